@@ -1,0 +1,138 @@
+/*
+ * wtconv.h - C ABI of the B200 (sm_100a) WTConv library.
+ *
+ * The operator is the wavelet convolution of Algorithm 1 (Sec. 2.1 of the paper):
+ *
+ *   X^0 = x
+ *   for l = 1..L:  Y^l = A X^(l-1)                 (2x2 orthonormal Haar analysis, Eq. 5)
+ *                  Z^l = s^l (.) (Y^l *dw W^l)      (k x k depthwise conv on the 4C subband channels, then scale)
+ *                  X^l = [Y^l]_LL                   (the raw low-pass band is carried down)
+ *   R^(L+1) = 0
+ *   for l = L..1:  R^l = A^T( ([Z^l]_LL + R^(l+1)) || [Z^l]_H )     (Haar synthesis)
+ *   out = s^0 (.) (x *dw W^0 + b) + R^1
+ *
+ * evaluated with the three exact reformulations of Sec. 4: the analysis butterfly is
+ * recomputed on chip (Sec. 4.1), the synthesis cascade is the bit-indexed closed form of
+ * Proposition 2 (Sec. 4.2), and the scales are folded into the weights (Eq. 8) with the
+ * gradients un-folded by Eq. 9 (Sec. 4.3).  The backward pass uses Sec. 2.2: the gradient
+ * of analysis is synthesis and vice versa.
+ *
+ * Conventions fixed where the paper is silent:
+ *   - "*dw" is a cross-correlation with zero padding R = k/2:
+ *         (X *dw W)[y,x] = sum_{u,v} W[u,v] X[y+u-R, x+v-R].
+ *   - An odd height/width is zero-padded on the bottom/right to even before each Haar
+ *     level: H_l = ceil(H_(l-1)/2); each synthesis result is cropped back.
+ *   - Subband order is (LL, LH, HL, HH); LH = (a+b-c-d)/2 carries the row sign, HL the
+ *     column sign, for the 2x2 block [a b; c d].
+ *
+ * Memory and execution contract (every entry point unless it says otherwise):
+ *   - Every pointer named "device" is a device pointer owned by the caller.  The library
+ *     never allocates, frees or synchronises; work is enqueued on `stream` and is complete
+ *     when the stream reaches that point.
+ *   - Activations (x, out, grad_out, grad_x) are contiguous [B][C][H][W] in `desc->dtype`,
+ *     base pointers 16-byte aligned.  Parameters and parameter gradients are float32 in
+ *     every mode; all arithmetic and accumulation is float32.
+ *       w0 [C][k][k]   s0 [C]   b0 [C] or NULL (no bias)
+ *       wl [L][C][4][k][k]   sl [L][C][4]      (ignored, may be NULL, when L == 0)
+ *   - Outputs are overwritten, never accumulated into.
+ *   - `workspace` is device scratch of at least the size wtconv_workspace_bytes reports,
+ *     256-byte aligned; its contents are undefined before and after a call.  Two calls
+ *     that overlap in time need distinct workspaces.
+ *   - Errors are returned as status codes before anything is launched; nothing traps or
+ *     aborts.  A failed launch is reported as WTCONV_ERR_CUDA.
+ */
+#ifndef WTCONV_H_
+#define WTCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { WTCONV_F32 = 0, WTCONV_F16 = 1, WTCONV_BF16 = 2 } wtconv_dtype;
+
+typedef enum {
+    WTCONV_OK = 0,
+    WTCONV_ERR_NULL = 1,        /* a required pointer is NULL */
+    WTCONV_ERR_SHAPE = 2,       /* B, C, H or W < 1, or the tensor exceeds 2^31-1 elements per plane set limits */
+    WTCONV_ERR_KERNEL_SIZE = 3, /* k not in {3, 5, 7} */
+    WTCONV_ERR_LEVELS = 4,      /* L outside [0, WTCONV_MAX_LEVELS] */
+    WTCONV_ERR_DTYPE = 5,
+    WTCONV_ERR_ALIGNMENT = 6,   /* an activation pointer is not 16-byte aligned, or workspace not 256-byte aligned */
+    WTCONV_ERR_WORKSPACE = 7,   /* workspace NULL or smaller than required */
+    WTCONV_ERR_ALIAS = 8,       /* an output overlaps an input */
+    WTCONV_ERR_ARCH = 9,        /* the current device is not compute capability 10.x */
+    WTCONV_ERR_CUDA = 10,       /* a CUDA runtime call or launch failed */
+    WTCONV_ERR_TIMEOUT = 11     /* reserved: a bounded device-side wait ran out */
+} wtconv_status;
+
+#define WTCONV_MAX_LEVELS 8
+
+/* desc->flags */
+#define WTCONV_FLAG_TILED_ONLY 1u /* never take the plane-resident kernels (used to test the tiled path) */
+
+typedef struct {
+    int32_t B, C, H, W; /* activation shape */
+    int32_t k;          /* depthwise kernel size: 3, 5 or 7 */
+    int32_t L;          /* decomposition levels, 0..WTCONV_MAX_LEVELS (0 = base path only) */
+    int32_t dtype;      /* wtconv_dtype of the activations */
+    uint32_t flags;
+} wtconv_desc;
+
+/* Static string for a status code (never NULL). */
+const char *wtconv_status_string(wtconv_status st);
+
+/* Level grid of Algorithm 1's Y^level: H_l = ceil(H / 2^level), same for W (level 0 = input).
+ * Pure host integer math; errors: NULL, LEVELS (level < 0 or > WTCONV_MAX_LEVELS), SHAPE. */
+wtconv_status wtconv_level_shape(const wtconv_desc *desc, int level, int32_t *Hl, int32_t *Wl);
+
+/* Scratch bytes wtconv_forward / wtconv_backward need for this descriptor (host call, no CUDA).
+ * Either output pointer may be NULL. */
+wtconv_status wtconv_workspace_bytes(const wtconv_desc *desc, size_t *fwd_bytes, size_t *bwd_bytes);
+
+/* Name of the kernel family a descriptor dispatches to ("plane" = whole-plane shared-memory
+ * kernels, "tiled" = per-level tiled kernels).  Host call; returns NULL for an invalid desc. */
+const char *wtconv_plan_name(const wtconv_desc *desc);
+
+/* Number of kernel launches one wtconv_forward / wtconv_backward call enqueues. */
+wtconv_status wtconv_launch_count(const wtconv_desc *desc, int32_t *fwd_launches, int32_t *bwd_launches);
+
+/* Forward pass of Algorithm 1 (device pointers).  out must not overlap x. */
+wtconv_status wtconv_forward(const wtconv_desc *desc, const void *x,
+                             const float *w0, const float *s0, const float *b0,
+                             const float *wl, const float *sl,
+                             void *out, void *workspace, size_t workspace_bytes, void *stream /* cudaStream_t */);
+
+/* Backward pass (device pointers): given grad_out = dLoss/d out, writes
+ *   grad_x [B][C][H][W] (dtype), grad_w0 [C][k][k], grad_s0 [C], grad_b0 [C] (NULL iff b0 is NULL),
+ *   grad_wl [L][C][4][k][k], grad_sl [L][C][4]      (float32; Eq. 9 already applied).
+ * Stateless: everything is recomputed from x, nothing saved by wtconv_forward is needed.
+ * grad_x must not overlap x or grad_out.  The batch reduction of the parameter gradients is
+ * deterministic (fixed-order partial sums, finished in float64). */
+wtconv_status wtconv_backward(const wtconv_desc *desc, const void *x, const void *grad_out,
+                              const float *w0, const float *s0, const float *b0,
+                              const float *wl, const float *sl,
+                              void *grad_x, float *grad_w0, float *grad_s0, float *grad_b0,
+                              float *grad_wl, float *grad_sl,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/* One training step from HOST memory: copies x, grad_out and the parameters to the device,
+ * runs wtconv_forward and wtconv_backward, and copies out, grad_x and the parameter
+ * gradients back, all asynchronously on `stream` (the host buffers should be pinned for the
+ * copies to overlap; they must stay valid until the stream reaches this point).
+ * Every h_* pointer is a HOST pointer with the layouts above; `workspace` is DEVICE scratch of
+ * at least wtconv_step_host_workspace_bytes.  h_b0 / h_grad_b0 may both be NULL. */
+wtconv_status wtconv_step_host_workspace_bytes(const wtconv_desc *desc, size_t *bytes);
+wtconv_status wtconv_step_host(const wtconv_desc *desc, const void *h_x, const void *h_grad_out,
+                               const float *h_w0, const float *h_s0, const float *h_b0,
+                               const float *h_wl, const float *h_sl,
+                               void *h_out, void *h_grad_x, float *h_grad_w0, float *h_grad_s0, float *h_grad_b0,
+                               float *h_grad_wl, float *h_grad_sl,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WTCONV_H_ */

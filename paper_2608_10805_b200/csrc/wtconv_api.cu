@@ -1,0 +1,434 @@
+// C ABI of the WTConv library: validation, workspace planning and kernel dispatch.
+// Declarations and the full contract are in include/wtconv.h.
+#include "../../include/wtconv.h"
+
+#include "common.cuh"
+#include "tiled_kernels.cuh"
+#include "plane_kernels.cuh"
+
+namespace {
+
+using wt::host_half_up;
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+struct Shapes {
+    int Hs[WTCONV_MAX_LEVELS + 1], Ws[WTCONV_MAX_LEVELS + 1];
+};
+
+wtconv_status validate_desc(const wtconv_desc *d) {
+    if (!d) return WTCONV_ERR_NULL;
+    if (d->B < 1 || d->C < 1 || d->H < 1 || d->W < 1) return WTCONV_ERR_SHAPE;
+    if ((int64_t)d->B * d->C > 0x7fffffffLL || (int64_t)d->H * d->W > 0x3fffffffLL) return WTCONV_ERR_SHAPE;
+    if (d->k != 3 && d->k != 5 && d->k != 7) return WTCONV_ERR_KERNEL_SIZE;
+    if (d->L < 0 || d->L > WTCONV_MAX_LEVELS) return WTCONV_ERR_LEVELS;
+    if (d->dtype != WTCONV_F32 && d->dtype != WTCONV_F16 && d->dtype != WTCONV_BF16) return WTCONV_ERR_DTYPE;
+    return WTCONV_OK;
+}
+
+Shapes level_shapes(const wtconv_desc *d) {
+    Shapes s;
+    s.Hs[0] = d->H;
+    s.Ws[0] = d->W;
+    for (int l = 1; l <= WTCONV_MAX_LEVELS; ++l) {
+        s.Hs[l] = host_half_up(s.Hs[l - 1]);
+        s.Ws[l] = host_half_up(s.Ws[l - 1]);
+    }
+    return s;
+}
+
+size_t elem_bytes(int dtype) { return dtype == WTCONV_F32 ? 4 : 2; }
+
+// ------------------------------------------------------------------ tiled-path workspace plan
+struct TiledPlan {
+    Shapes sh;
+    int P, KK;
+    // forward
+    size_t z_off[WTCONV_MAX_LEVELS], xc_off[WTCONV_MAX_LEVELS];  // Z^l / dY^l and carrier X^l (index l-1)
+    size_t fwd_bytes;
+    // backward extras
+    size_t gc_off[WTCONV_MAX_LEVELS];
+    size_t part0_off, partl_off[WTCONV_MAX_LEVELS];
+    int bsplit0, np0, bsplitl[WTCONV_MAX_LEVELS], npl[WTCONV_MAX_LEVELS];
+    int tx0, ty0, txl[WTCONV_MAX_LEVELS], tyl[WTCONV_MAX_LEVELS];
+    size_t bwd_bytes;
+};
+
+int pick_bsplit(int B, long long blocks_per_batchloop) {
+    // enough blocks to fill 148 SMs several times over, but never more than one batch per block
+    long long want = (4LL * 148 * 2 + blocks_per_batchloop - 1) / blocks_per_batchloop;
+    if (want < 1) want = 1;
+    if (want > B) want = B;
+    return (int)want;
+}
+
+TiledPlan make_tiled_plan(const wtconv_desc *d) {
+    TiledPlan p;
+    p.sh = level_shapes(d);
+    p.P = d->B * d->C;
+    p.KK = d->k * d->k;
+    size_t off = 0;
+    for (int l = 1; l <= d->L; ++l) {
+        size_t S = (size_t)p.sh.Hs[l] * p.sh.Ws[l];
+        p.z_off[l - 1] = off;
+        off = align_up(off + sizeof(float) * 4 * S * p.P);
+        p.xc_off[l - 1] = off;
+        if (l < d->L) off = align_up(off + sizeof(float) * S * p.P);
+    }
+    p.fwd_bytes = off;
+    for (int l = 1; l < d->L; ++l) {
+        size_t S = (size_t)p.sh.Hs[l] * p.sh.Ws[l];
+        p.gc_off[l - 1] = off;
+        off = align_up(off + sizeof(float) * S * p.P);
+    }
+    p.tx0 = cdiv(d->W, wt::tiled::TW);
+    p.ty0 = cdiv(d->H, wt::tiled::TH);
+    p.bsplit0 = pick_bsplit(d->B, (long long)p.tx0 * p.ty0 * d->C);
+    p.np0 = p.tx0 * p.ty0 * p.bsplit0;
+    p.part0_off = off;
+    off = align_up(off + sizeof(float) * (size_t)d->C * p.np0 * (p.KK + 1));
+    for (int l = 1; l <= d->L; ++l) {
+        p.txl[l - 1] = cdiv(p.sh.Ws[l], wt::tiled::TW);
+        p.tyl[l - 1] = cdiv(p.sh.Hs[l], wt::tiled::TH);
+        p.bsplitl[l - 1] = pick_bsplit(d->B, (long long)p.txl[l - 1] * p.tyl[l - 1] * d->C);
+        p.npl[l - 1] = p.txl[l - 1] * p.tyl[l - 1] * p.bsplitl[l - 1];
+        p.partl_off[l - 1] = off;
+        off = align_up(off + sizeof(float) * (size_t)d->C * p.npl[l - 1] * 4 * p.KK);
+    }
+    p.bwd_bytes = off;
+    return p;
+}
+
+bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
+    const char *pa = (const char *)a, *pb = (const char *)b;
+    return pa < pb + nb && pb < pa + na;
+}
+
+wtconv_status check_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WTCONV_ERR_CUDA;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return WTCONV_ERR_CUDA;
+    return major == 10 ? WTCONV_OK : WTCONV_ERR_ARCH;
+}
+
+inline wtconv_status launch_status() { return cudaGetLastError() == cudaSuccess ? WTCONV_OK : WTCONV_ERR_CUDA; }
+
+// ------------------------------------------------------------------ tiled forward / backward
+template <typename T, int K>
+wtconv_status tiled_forward(const wtconv_desc *d, const T *x, const float *w0, const float *s0, const float *b0,
+                            const float *wl, const float *sl, T *out, char *ws, cudaStream_t st) {
+    using namespace wt::tiled;
+    TiledPlan pl = make_tiled_plan(d);
+    wt::tiled::LevelPtrs lv = {};
+    const int C = d->C, KK = K * K;
+    for (int l = 1; l <= d->L; ++l) {
+        const int Hp = pl.sh.Hs[l - 1], Wp = pl.sh.Ws[l - 1], Hl = pl.sh.Hs[l], Wl = pl.sh.Ws[l];
+        float *Z = (float *)(ws + pl.z_off[l - 1]);
+        float *Xl = (l < d->L) ? (float *)(ws + pl.xc_off[l - 1]) : nullptr;
+        dim3 grid(pl.P, cdiv(Wl, TW), cdiv(Hl, TH));
+        const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
+        if (l == 1)
+            level_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, Hp, Wp, Hl, Wl, C, wq, sq, Z, Xl);
+        else
+            level_fwd_kernel<float, K><<<grid, NTHREADS, 0, st>>>((const float *)(ws + pl.xc_off[l - 2]), Hp, Wp, Hl,
+                                                                   Wl, C, wq, sq, Z, Xl);
+        lv.z[l - 1] = Z;
+        lv.Hl[l - 1] = Hl;
+        lv.Wl[l - 1] = Wl;
+    }
+    dim3 grid(pl.P, cdiv(d->W, TW), cdiv(d->H, TH));
+    synth_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, d->H, d->W, C, d->L, w0, s0, b0, lv, out);
+    return launch_status();
+}
+
+wtconv_status launch_epilogue(const wtconv_desc *d, const wt::EpiloguePtrs &ep, const float *w0, const float *s0,
+                              const float *b0, const float *wl, const float *sl, float *gw0, float *gs0, float *gb0,
+                              float *gwl, float *gsl, cudaStream_t st) {
+    const int KK = d->k * d->k;
+    size_t smem = sizeof(double) * (KK + 1 + (size_t)d->L * 4 * KK);
+    wt::unfold_epilogue_kernel<<<d->C, 128, smem, st>>>(d->C, d->k, d->L, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl,
+                                                        gsl);
+    return launch_status();
+}
+
+template <typename T, int K>
+wtconv_status tiled_backward(const wtconv_desc *d, const T *x, const T *g, const float *w0, const float *s0,
+                             const float *b0, const float *wl, const float *sl, T *gx, float *gw0, float *gs0,
+                             float *gb0, float *gwl, float *gsl, char *ws, cudaStream_t st) {
+    using namespace wt::tiled;
+    TiledPlan pl = make_tiled_plan(d);
+    wt::tiled::LevelPtrs lv = {};
+    wt::EpiloguePtrs ep = {};
+    const int C = d->C, KK = K * K;
+    for (int l = 1; l <= d->L; ++l) {
+        const int Hp = pl.sh.Hs[l - 1], Wp = pl.sh.Ws[l - 1], Hl = pl.sh.Hs[l], Wl = pl.sh.Ws[l];
+        float *dY = (float *)(ws + pl.z_off[l - 1]);
+        float *Xl = (l < d->L) ? (float *)(ws + pl.xc_off[l - 1]) : nullptr;
+        float *Gl = (l < d->L) ? (float *)(ws + pl.gc_off[l - 1]) : nullptr;
+        float *part = (float *)(ws + pl.partl_off[l - 1]);
+        dim3 grid(C * pl.bsplitl[l - 1], pl.txl[l - 1], pl.tyl[l - 1]);
+        const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
+        if (l == 1)
+            level_bwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, g, Hp, Wp, Hl, Wl, d->B, C, pl.bsplitl[l - 1], wq, sq,
+                                                              dY, Xl, Gl, part);
+        else
+            level_bwd_kernel<float, K><<<grid, NTHREADS, 0, st>>>(
+                (const float *)(ws + pl.xc_off[l - 2]), (const float *)(ws + pl.gc_off[l - 2]), Hp, Wp, Hl, Wl, d->B, C,
+                pl.bsplitl[l - 1], wq, sq, dY, Xl, Gl, part);
+        lv.z[l - 1] = dY;
+        lv.Hl[l - 1] = Hl;
+        lv.Wl[l - 1] = Wl;
+        ep.partl[l - 1] = part;
+        ep.npl[l - 1] = pl.npl[l - 1];
+    }
+    float *part0 = (float *)(ws + pl.part0_off);
+    dim3 grid(C * pl.bsplit0, pl.tx0, pl.ty0);
+    synth_bwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, g, d->H, d->W, d->B, C, d->L, pl.bsplit0, w0, s0, lv, gx,
+                                                      part0);
+    ep.part0 = part0;
+    ep.np0 = pl.np0;
+    if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
+    return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
+}
+
+// ------------------------------------------------------------------ dispatch
+bool use_plane_path(const wtconv_desc *d) {
+    if (d->flags & WTCONV_FLAG_TILED_ONLY) return false;
+    return wt::plane::supported(d->H, d->W, d->k, d->L, d->dtype);
+}
+
+template <typename T, int K>
+wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, const float *s0, const float *b0,
+                         const float *wl, const float *sl, void *out, char *ws, cudaStream_t st) {
+    if (use_plane_path(d)) {
+        if constexpr (K == 5)
+            return wt::plane::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws,
+                                         st) == cudaSuccess
+                       ? WTCONV_OK
+                       : WTCONV_ERR_CUDA;
+    }
+    return tiled_forward<T, K>(d, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st);
+}
+
+template <typename T, int K>
+wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, const float *w0, const float *s0,
+                          const float *b0, const float *wl, const float *sl, void *gx, float *gw0, float *gs0,
+                          float *gb0, float *gwl, float *gsl, char *ws, cudaStream_t st) {
+    if (use_plane_path(d)) {
+        if constexpr (K == 5) {
+            wt::EpiloguePtrs ep = {};
+            if (wt::plane::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl,
+                                       (T *)gx, ws, &ep, st) != cudaSuccess)
+                return WTCONV_ERR_CUDA;
+            return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
+        }
+    }
+    return tiled_backward<T, K>(d, (const T *)x, (const T *)g, w0, s0, b0, wl, sl, (T *)gx, gw0, gs0, gb0, gwl, gsl,
+                                ws, st);
+}
+
+#define WT_DISPATCH(FN, ...)                                                                   \
+    do {                                                                                       \
+        switch (d->dtype * 8 + d->k) {                                                         \
+            case WTCONV_F32 * 8 + 3: return FN<float, 3>(__VA_ARGS__);                         \
+            case WTCONV_F32 * 8 + 5: return FN<float, 5>(__VA_ARGS__);                         \
+            case WTCONV_F32 * 8 + 7: return FN<float, 7>(__VA_ARGS__);                         \
+            case WTCONV_F16 * 8 + 3: return FN<__half, 3>(__VA_ARGS__);                        \
+            case WTCONV_F16 * 8 + 5: return FN<__half, 5>(__VA_ARGS__);                        \
+            case WTCONV_F16 * 8 + 7: return FN<__half, 7>(__VA_ARGS__);                        \
+            case WTCONV_BF16 * 8 + 3: return FN<__nv_bfloat16, 3>(__VA_ARGS__);                \
+            case WTCONV_BF16 * 8 + 5: return FN<__nv_bfloat16, 5>(__VA_ARGS__);                \
+            case WTCONV_BF16 * 8 + 7: return FN<__nv_bfloat16, 7>(__VA_ARGS__);                \
+        }                                                                                      \
+        return WTCONV_ERR_DTYPE;                                                               \
+    } while (0)
+
+size_t fwd_ws_bytes(const wtconv_desc *d) {
+    if (use_plane_path(d)) return align_up(wt::plane::forward_workspace_bytes(d->B, d->C, d->H, d->W, d->L));
+    return make_tiled_plan(d).fwd_bytes;
+}
+size_t bwd_ws_bytes(const wtconv_desc *d) {
+    if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L));
+    return make_tiled_plan(d).bwd_bytes;
+}
+
+struct ParamSizes {
+    size_t w0, s0, wl, sl;
+};
+ParamSizes param_sizes(const wtconv_desc *d) {
+    size_t KK = (size_t)d->k * d->k, C = d->C, L = d->L;
+    return {C * KK * 4, C * 4, L * C * 4 * KK * 4, L * C * 4 * 4};
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *wtconv_status_string(wtconv_status st) {
+    switch (st) {
+        case WTCONV_OK: return "ok";
+        case WTCONV_ERR_NULL: return "a required pointer is NULL";
+        case WTCONV_ERR_SHAPE: return "invalid shape";
+        case WTCONV_ERR_KERNEL_SIZE: return "kernel size must be 3, 5 or 7";
+        case WTCONV_ERR_LEVELS: return "level count out of range";
+        case WTCONV_ERR_DTYPE: return "unknown dtype";
+        case WTCONV_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+        case WTCONV_ERR_WORKSPACE: return "workspace missing or too small";
+        case WTCONV_ERR_ALIAS: return "an output overlaps an input";
+        case WTCONV_ERR_ARCH: return "device is not compute capability 10.x";
+        case WTCONV_ERR_CUDA: return "CUDA runtime error";
+        case WTCONV_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+wtconv_status wtconv_level_shape(const wtconv_desc *d, int level, int32_t *Hl, int32_t *Wl) {
+    if (!d || !Hl || !Wl) return WTCONV_ERR_NULL;
+    if (d->H < 1 || d->W < 1) return WTCONV_ERR_SHAPE;
+    if (level < 0 || level > WTCONV_MAX_LEVELS) return WTCONV_ERR_LEVELS;
+    Shapes s = level_shapes(d);
+    *Hl = s.Hs[level];
+    *Wl = s.Ws[level];
+    return WTCONV_OK;
+}
+
+wtconv_status wtconv_workspace_bytes(const wtconv_desc *d, size_t *fwd_bytes, size_t *bwd_bytes) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (fwd_bytes) *fwd_bytes = fwd_ws_bytes(d);
+    if (bwd_bytes) *bwd_bytes = bwd_ws_bytes(d);
+    return WTCONV_OK;
+}
+
+const char *wtconv_plan_name(const wtconv_desc *d) {
+    if (validate_desc(d) != WTCONV_OK) return nullptr;
+    return use_plane_path(d) ? "plane" : "tiled";
+}
+
+wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *bwd) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (use_plane_path(d)) {
+        if (fwd) *fwd = 1;
+        if (bwd) *bwd = 2;
+    } else {
+        if (fwd) *fwd = d->L + 1;
+        if (bwd) *bwd = d->L + 2;
+    }
+    return WTCONV_OK;
+}
+
+wtconv_status wtconv_forward(const wtconv_desc *d, const void *x, const float *w0, const float *s0, const float *b0,
+                             const float *wl, const float *sl, void *out, void *workspace, size_t workspace_bytes,
+                             void *stream) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (!x || !w0 || !s0 || !out || (d->L > 0 && (!wl || !sl))) return WTCONV_ERR_NULL;
+    if (((uintptr_t)x | (uintptr_t)out) & 15) return WTCONV_ERR_ALIGNMENT;
+    const size_t need = fwd_ws_bytes(d);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return WTCONV_ERR_WORKSPACE;
+    if (need > 0 && ((uintptr_t)workspace & (ALIGN - 1))) return WTCONV_ERR_ALIGNMENT;
+    const size_t nbytes = (size_t)d->B * d->C * d->H * d->W * elem_bytes(d->dtype);
+    if (overlaps(x, nbytes, out, nbytes)) return WTCONV_ERR_ALIAS;
+    if ((st = check_device()) != WTCONV_OK) return st;
+    char *ws = (char *)workspace;
+    cudaStream_t cs = (cudaStream_t)stream;
+    WT_DISPATCH(forward_tk, d, x, w0, s0, b0, wl, sl, out, ws, cs);
+}
+
+wtconv_status wtconv_backward(const wtconv_desc *d, const void *x, const void *grad_out, const float *w0,
+                              const float *s0, const float *b0, const float *wl, const float *sl, void *grad_x,
+                              float *grad_w0, float *grad_s0, float *grad_b0, float *grad_wl, float *grad_sl,
+                              void *workspace, size_t workspace_bytes, void *stream) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (!x || !grad_out || !w0 || !s0 || !grad_x || !grad_w0 || !grad_s0) return WTCONV_ERR_NULL;
+    if (d->L > 0 && (!wl || !sl || !grad_wl || !grad_sl)) return WTCONV_ERR_NULL;
+    if ((b0 == nullptr) != (grad_b0 == nullptr)) return WTCONV_ERR_NULL;
+    if (((uintptr_t)x | (uintptr_t)grad_out | (uintptr_t)grad_x) & 15) return WTCONV_ERR_ALIGNMENT;
+    const size_t need = bwd_ws_bytes(d);
+    if (!workspace || workspace_bytes < need) return WTCONV_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
+    const size_t nbytes = (size_t)d->B * d->C * d->H * d->W * elem_bytes(d->dtype);
+    if (overlaps(x, nbytes, grad_x, nbytes) || overlaps(grad_out, nbytes, grad_x, nbytes)) return WTCONV_ERR_ALIAS;
+    if ((st = check_device()) != WTCONV_OK) return st;
+    char *ws = (char *)workspace;
+    cudaStream_t cs = (cudaStream_t)stream;
+    WT_DISPATCH(backward_tk, d, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad_s0, grad_b0, grad_wl, grad_sl,
+                ws, cs);
+}
+
+// Device staging layout of wtconv_step_host: x, g, out, gx (activation dtype), then the
+// parameters, then the parameter gradients, then the kernels' own workspace.
+wtconv_status wtconv_step_host_workspace_bytes(const wtconv_desc *d, size_t *bytes) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (!bytes) return WTCONV_ERR_NULL;
+    const size_t act = align_up((size_t)d->B * d->C * d->H * d->W * elem_bytes(d->dtype));
+    ParamSizes ps = param_sizes(d);
+    const size_t par = align_up(ps.w0) + 2 * align_up(ps.s0) + align_up(ps.wl) + align_up(ps.sl);
+    size_t f = fwd_ws_bytes(d), b = bwd_ws_bytes(d);
+    *bytes = 4 * act + 2 * par + (f > b ? f : b);
+    return WTCONV_OK;
+}
+
+wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void *h_g, const float *h_w0,
+                               const float *h_s0, const float *h_b0, const float *h_wl, const float *h_sl, void *h_out,
+                               void *h_gx, float *h_gw0, float *h_gs0, float *h_gb0, float *h_gwl, float *h_gsl,
+                               void *workspace, size_t workspace_bytes, void *stream) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (!h_x || !h_g || !h_w0 || !h_s0 || !h_out || !h_gx || !h_gw0 || !h_gs0) return WTCONV_ERR_NULL;
+    if (d->L > 0 && (!h_wl || !h_sl || !h_gwl || !h_gsl)) return WTCONV_ERR_NULL;
+    if ((h_b0 == nullptr) != (h_gb0 == nullptr)) return WTCONV_ERR_NULL;
+    size_t need = 0;
+    wtconv_step_host_workspace_bytes(d, &need);
+    if (!workspace || workspace_bytes < need) return WTCONV_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
+    cudaStream_t cs = (cudaStream_t)stream;
+    const size_t act_raw = (size_t)d->B * d->C * d->H * d->W * elem_bytes(d->dtype), act = align_up(act_raw);
+    ParamSizes ps = param_sizes(d);
+    char *p = (char *)workspace;
+    char *dx_ = p, *dg = p + act, *dout = p + 2 * act, *dgx = p + 3 * act;
+    p += 4 * act;
+    auto take = [&](size_t n) { char *q = p; p += align_up(n); return q; };
+    float *w0 = (float *)take(ps.w0), *s0 = (float *)take(ps.s0), *b0 = (float *)take(ps.s0);
+    float *wl = (float *)take(ps.wl), *sl = (float *)take(ps.sl);
+    float *gw0 = (float *)take(ps.w0), *gs0 = (float *)take(ps.s0), *gb0 = (float *)take(ps.s0);
+    float *gwl = (float *)take(ps.wl), *gsl = (float *)take(ps.sl);
+    const size_t rest = workspace_bytes - (size_t)(p - (char *)workspace);
+    bool ok = true;
+    auto h2d = [&](void *dst, const void *src, size_t n) {
+        if (n) ok = ok && cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+    };
+    auto d2h = [&](void *dst, const void *src, size_t n) {
+        if (n) ok = ok && cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, cs) == cudaSuccess;
+    };
+    h2d(dx_, h_x, act_raw);
+    h2d(dg, h_g, act_raw);
+    h2d(w0, h_w0, ps.w0);
+    h2d(s0, h_s0, ps.s0);
+    if (h_b0) h2d(b0, h_b0, ps.s0);
+    h2d(wl, h_wl, ps.wl);
+    h2d(sl, h_sl, ps.sl);
+    if (!ok) return WTCONV_ERR_CUDA;
+    const float *b0p = h_b0 ? b0 : nullptr;
+    st = wtconv_forward(d, dx_, w0, s0, b0p, wl, sl, dout, p, rest, stream);
+    if (st != WTCONV_OK) return st;
+    st = wtconv_backward(d, dx_, dg, w0, s0, b0p, wl, sl, dgx, gw0, gs0, h_b0 ? gb0 : nullptr, gwl, gsl, p, rest,
+                         stream);
+    if (st != WTCONV_OK) return st;
+    d2h(h_out, dout, act_raw);
+    d2h(h_gx, dgx, act_raw);
+    d2h(h_gw0, gw0, ps.w0);
+    d2h(h_gs0, gs0, ps.s0);
+    if (h_b0) d2h(h_gb0, gb0, ps.s0);
+    d2h(h_gwl, gwl, ps.wl);
+    d2h(h_gsl, gsl, ps.sl);
+    return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,88 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and rejects bad arguments with the documented status codes before any launch."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_10805_b200 import build as wbuild
+from paper_2608_10805_b200 import wtconv as wt
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    wbuild.build()
+    return wt.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "wtconv.h")).read()
+    declared = set(re.findall(r"\b(wtconv_[a-z_0-9]+)\s*\(", hdr))
+    assert declared == set(wt.EXPORTS), declared ^ set(wt.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    for code in range(0, 12):
+        s = lib.wtconv_status_string(code)
+        assert s and s != b"unknown status"
+    assert lib.wtconv_status_string(99) == b"unknown status"
+
+
+def test_level_shape_and_errors(lib):
+    d = wt.make_desc(1, 1, 225, 225, 5, 5, "f16")
+    assert [wt.wtconv_level_shape(d, l) for l in range(6)] == [(225, 225), (113, 113), (57, 57), (29, 29), (15, 15), (8, 8)]
+    with pytest.raises(wt.WTConvError) as e:
+        wt.wtconv_level_shape(d, 9)
+    assert e.value.code == 4
+
+
+@pytest.mark.parametrize("kw,code", [(dict(B=0), 2), (dict(H=0), 2), (dict(k=4), 3), (dict(k=9), 3), (dict(L=-1), 4),
+                                     (dict(L=9), 4), (dict(dtype=7), 5)])
+def test_descriptor_validation(lib, kw, code):
+    base = dict(B=2, C=3, H=8, W=8, k=5, L=2, dtype=0, flags=0)
+    base.update(kw)
+    d = wt.Desc(**base)
+    f, b = ctypes.c_size_t(), ctypes.c_size_t()
+    assert lib.wtconv_workspace_bytes(ctypes.byref(d), ctypes.byref(f), ctypes.byref(b)) == code
+    assert wt.wtconv_plan_name(d) is None
+
+
+def test_argument_validation_happens_before_any_cuda_call(lib):
+    d = wt.make_desc(2, 3, 8, 8, 5, 2, "f32")
+    fb, bb = wt.wtconv_workspace_bytes(d)
+    assert fb > 0 and bb >= fb
+    buf = (ctypes.c_char * 4096)()
+    a = ctypes.addressof(buf)
+    a = (a + 255) // 256 * 256
+    P = ctypes.c_void_p
+    # NULL x
+    assert lib.wtconv_forward(ctypes.byref(d), None, P(a), P(a), None, P(a), P(a), P(a + 1024), P(a), fb, None) == 1
+    # misaligned activation pointer
+    assert lib.wtconv_forward(ctypes.byref(d), P(a + 4), P(a), P(a), None, P(a), P(a), P(a + 2048), P(a), fb, None) == 6
+    # workspace too small
+    assert lib.wtconv_forward(ctypes.byref(d), P(a), P(a), P(a), None, P(a), P(a), P(a + 2048), P(a), fb - 1, None) == 7
+    # out overlaps x
+    assert lib.wtconv_forward(ctypes.byref(d), P(a), P(a), P(a), None, P(a), P(a), P(a + 16), P(a), fb, None) == 8
+    # backward: bias and its gradient must come together
+    args = [P(a), P(a), P(a), P(a), P(a), P(a), P(a), P(a + 2048), P(a), P(a), None, P(a), P(a)]
+    assert lib.wtconv_backward(ctypes.byref(d), *args, P(a), bb, None) == 1
+
+
+def test_plan_and_launch_count(lib):
+    d = wt.make_desc(2, 3, 300, 300, 5, 3, "f32")
+    assert wt.wtconv_plan_name(d) == "tiled"
+    assert wt.wtconv_launch_count(d) == (4, 5)
+    dt = wt.make_desc(2, 3, 56, 56, 5, 3, "f32", wt.FLAG_TILED_ONLY)
+    assert wt.wtconv_plan_name(dt) == "tiled"
+
+
+def test_binding_refuses_to_run_without_the_library(monkeypatch):
+    monkeypatch.setattr(wt, "_lib", None)
+    monkeypatch.setattr(wt, "LIB_PATH", "/nonexistent/libwtconv_b200.so")
+    with pytest.raises(OSError):
+        wt.lib()
