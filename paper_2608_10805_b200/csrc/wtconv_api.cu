@@ -206,7 +206,7 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
     if (use_plane_path(d)) {
         if constexpr (K == 5)
             return wt::plane::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws,
-                                         st) == cudaSuccess
+                                         st, d->flags >> 8) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
@@ -221,7 +221,7 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
         if constexpr (K == 5) {
             wt::EpiloguePtrs ep = {};
             if (wt::plane::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl,
-                                       (T *)gx, ws, &ep, st) != cudaSuccess)
+                                       (T *)gx, ws, &ep, st, d->flags >> 8) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
         }
@@ -251,7 +251,7 @@ size_t fwd_ws_bytes(const wtconv_desc *d) {
     return make_tiled_plan(d).fwd_bytes;
 }
 size_t bwd_ws_bytes(const wtconv_desc *d) {
-    if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L));
+    if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, d->flags >> 8));
     return make_tiled_plan(d).bwd_bytes;
 }
 
@@ -313,7 +313,7 @@ wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *b
     if (st != WTCONV_OK) return st;
     if (use_plane_path(d)) {
         if (fwd) *fwd = 1;
-        if (bwd) *bwd = 2;
+        if (bwd) *bwd = 3; /* weight-gradient, input-gradient, epilogue (plus one memset node) */
     } else {
         if (fwd) *fwd = d->L + 1;
         if (bwd) *bwd = d->L + 2;
