@@ -80,6 +80,18 @@ __device__ __forceinline__ Haar4x2 haar2(u64 a, u64 b, u64 c, u64 d) {
 }
 
 // ------------------------------------------------------------------ geometry (host-planned, passed by value)
+// Division by a launch-invariant divisor as multiply-high: exact while dividend * divisor < 2^32.
+struct FastDiv {
+    unsigned mul, d;
+};
+inline FastDiv make_fastdiv(int d) {
+    FastDiv f;
+    f.d = (unsigned)(d < 1 ? 1 : d);
+    f.mul = (unsigned)(0x100000000ULL / f.d) + 1u;
+    return f;
+}
+__device__ __forceinline__ int fdiv(int e, const FastDiv &f) { return f.d == 1 ? e : (int)__umulhi((unsigned)e, f.mul); }
+
 struct Geom {
     int B, C, H, W, L;
     int Hl[MAXL + 1], Wl[MAXL + 1];        // level grids, index 0 = input
@@ -93,10 +105,15 @@ struct Geom {
     int tx[MAXL + 1], ty[MAXL + 1];        // 4x4 tiles per level grid (index 0 = base)
     int lvl_start[MAXL + 2];               // per pair: first level-item of level l (1..L); [L+1] = count
     int nbase;                             // base tiles per pair
-    int wtab_off;                          // offset of the folded weight table [(1+4L)*25 + 1] float2
+    int wtab_off;                          // offset of the folded weight table [(1+4L)][26] float2 (+ bias entry)
     int smem_u64;                          // shared memory in float2 units
     int bgroups, ncp, units;               // work units = ncp channel pairs x bgroups image groups
     int nthreads, nblocks, blocks_per_sm;
+    int vec;                               // 1: W % 4 == 0, rows can be staged with 4-element vector loads
+    int npatch;                            // staging work items per pair (vec: 2x4 pixel patches, else 2x2 blocks)
+    FastDiv d_npatch, d_prow;              // / npatch, / (patches per patch-row)
+    FastDiv d_lvl[MAXL + 1], d_lvlw[MAXL + 1];  // / (Hl*Wl), / Wl   (levels >= 2 staging)
+    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase;
     // weight-gradient kernel: class-major thread allocation and partial-sum slots
     int thr_start[4 * MAXL + 2];
     int np;
@@ -110,8 +127,17 @@ __host__ __device__ inline int block_of_unit(long long v, int nb, int units) {
     return (int)(((v + 1) * nb - 1) / units);
 }
 
+// Shared-memory layout of a haloed array row (pitch float2, pitch % 4 == 0): the 16-byte chunks
+// (two float2) of a row are de-interleaved, even chunks in the first half of the row and odd chunks in
+// the second.  A thread's 4x4 tile window starts at column 4*tx, so lanes of a warp read chunk
+// 2*tx + j: for fixed j consecutive lanes hit consecutive 16-byte words - no bank conflicts.
+__device__ __forceinline__ int phys_col(int col, int half) {
+    return ((col >> 1) & 1) * half + ((col >> 2) << 1) + (col & 1);
+}
+
+constexpr int WT_STRIDE = 26;  // float2 per class in the weight table (25 taps, padded to 16 bytes)
+
 // ------------------------------------------------------------------ shared device pieces
-template <typename T>
 __device__ __forceinline__ void build_weight_table(u64 *wtab, const Geom &g, int cA, bool hasB, bool flip,
                                                    const float *__restrict__ w0, const float *__restrict__ s0,
                                                    const float *__restrict__ b0, const float *__restrict__ wl,
@@ -129,7 +155,7 @@ __device__ __forceinline__ void build_weight_table(u64 *wtab, const Geom &g, int
             wa = __ldg(wl + ia * KK + src) * __ldg(sl + ia);
             if (hasB) wb = __ldg(wl + ib * KK + src) * __ldg(sl + ib);
         }
-        wtab[e] = pk(wa, wb);  // Eq. 8: scale folded into the weight
+        wtab[cls * WT_STRIDE + t] = pk(wa, wb);  // Eq. 8: scale folded into the weight
     }
     if (threadIdx.x == 0) {
         float ba = 0.f, bb = 0.f;
@@ -137,18 +163,52 @@ __device__ __forceinline__ void build_weight_table(u64 *wtab, const Geom &g, int
             ba = __ldg(s0 + cA) * __ldg(b0 + cA);
             if (hasB) bb = __ldg(s0 + cB) * __ldg(b0 + cB);
         }
-        wtab[ncls * KK] = pk(ba, bb);
+        wtab[KK] = pk(ba, bb);  // the spare 26th entry of class 0
     }
 }
 
-// Stage the planes of one unit: x into the haloed array `off[0]` and its level-1 Haar subbands into
-// `off[1]` (both planes of each pair interleaved).  Pixels beyond H x W are never written and stay
+__device__ __forceinline__ void load_weights(const u64 *wt, u64 (&w)[KK]) {
+    const ulonglong2 *q = reinterpret_cast<const ulonglong2 *>(wt);
+#pragma unroll
+    for (int t = 0; t < 12; ++t) {
+        const ulonglong2 v = q[t];
+        w[2 * t] = v.x;
+        w[2 * t + 1] = v.y;
+    }
+    w[24] = wt[24];
+}
+
+template <typename T>
+__device__ __forceinline__ void load4(const T *p, float (&v)[4]);
+template <>
+__device__ __forceinline__ void load4<float>(const float *p, float (&v)[4]) {
+    const float4 q = __ldg(reinterpret_cast<const float4 *>(p));
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+}
+template <>
+__device__ __forceinline__ void load4<__half>(const __half *p, float (&v)[4]) {
+    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+template <>
+__device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16 *p, float (&v)[4]) {
+    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.y));
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+
+// Stage the planes of one unit: x into the haloed array `off[0]` and its level-1 Haar subbands (Eq. 5)
+// into `off[1]`, both planes of each pair interleaved.  Pixels beyond H x W are never written and stay
 // zero (odd-size padding and conv halo); images beyond the batch are written as zeros.
 template <typename T>
-__device__ __forceinline__ void stage_level1(u64 *sm, const Geom &g, const int *off, const T *__restrict__ x, int cA,
-                                             bool hasB, int bg) {
+__device__ __forceinline__ void stage_input(u64 *sm, const Geom &g, const int *off, const T *__restrict__ x, int cA,
+                                            bool hasB, int bg) {
     const int H = g.H, W = g.W;
     const size_t HW = (size_t)H * W;
+    const int p0 = g.pitch[0], h0 = p0 >> 1;
     if (g.L == 0) {
         for (int e = threadIdx.x; e < g.NPP * H * W; e += blockDim.x) {
             const int slot = e / (H * W), r = e - slot * (H * W), y = r / W, xx = r - y * W;
@@ -159,14 +219,59 @@ __device__ __forceinline__ void stage_level1(u64 *sm, const Geom &g, const int *
                 va = ldf(pa);
                 if (hasB) vb = ldf(pa + HW);
             }
-            sm[(size_t)slot * g.slot_stride + off[0] + (y + 2) * g.pitch[0] + xx + 2] = pk(va, vb);
+            sm[(size_t)slot * g.slot_stride + off[0] + (y + 2) * p0 + phys_col(xx + 2, h0)] = pk(va, vb);
         }
         return;
     }
-    const int H1 = g.Hl[1], W1 = g.Wl[1], nblk = H1 * W1;
-    const int p0 = g.pitch[0], p1 = g.pitch[1], sub1 = g.rows[1] * p1;
-    for (int e = threadIdx.x; e < g.NPP * nblk; e += blockDim.x) {
-        const int slot = e / nblk, r = e - slot * nblk, i = r / W1, j = r - i * W1;
+    const int p1 = g.pitch[1], h1 = p1 >> 1, sub1 = g.rows[1] * p1;
+    if (g.vec) {
+        // work item = 2 rows x 4 columns of both planes: two Haar blocks, whole 16-byte chunks everywhere
+        for (int e = threadIdx.x; e < g.NPP * g.npatch; e += blockDim.x) {
+            const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
+            const int i = fdiv(r, g.d_prow), q = r - i * (int)g.d_prow.d;
+            const int b = bg * g.NPP + slot, y = 2 * i;
+            const bool y1 = y + 1 < H;
+            float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f}, b0[4] = {0.f, 0.f, 0.f, 0.f},
+                  b1[4] = {0.f, 0.f, 0.f, 0.f};
+            if (b < g.B) {
+                const T *pa = x + ((size_t)b * g.C + cA) * HW + (size_t)y * W + 4 * q;
+                load4<T>(pa, a0);
+                if (y1) load4<T>(pa + W, a1);
+                if (hasB) {
+                    load4<T>(pa + HW, b0);
+                    if (y1) load4<T>(pa + HW + W, b1);
+                }
+            }
+            u64 *S = sm + (size_t)slot * g.slot_stride;
+            u64 r0v[4], r1v[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                r0v[c] = pk(a0[c], b0[c]);
+                r1v[c] = pk(a1[c], b1[c]);
+            }
+            // columns 4q+2 .. 4q+5 = chunk 2q+1 (odd half, index q) and chunk 2q+2 (even half, index q+1)
+            u64 *X = S + off[0] + (y + 2) * p0;
+            *reinterpret_cast<ulonglong2 *>(X + h0 + 2 * q) = make_ulonglong2(r0v[0], r0v[1]);
+            *reinterpret_cast<ulonglong2 *>(X + 2 * q + 2) = make_ulonglong2(r0v[2], r0v[3]);
+            if (y1) {
+                *reinterpret_cast<ulonglong2 *>(X + p0 + h0 + 2 * q) = make_ulonglong2(r1v[0], r1v[1]);
+                *reinterpret_cast<ulonglong2 *>(X + p0 + 2 * q + 2) = make_ulonglong2(r1v[2], r1v[3]);
+            }
+            const Haar4x2 ha = haar2(r0v[0], r0v[1], r1v[0], r1v[1]), hb = haar2(r0v[2], r0v[3], r1v[2], r1v[3]);
+            // level-1 columns 2q+2, 2q+3 = chunk q+1
+            u64 *Y = S + off[1] + (i + 2) * p1 + ((q + 1) & 1) * h1 + ((q + 1) >> 1) * 2;
+            *reinterpret_cast<ulonglong2 *>(Y) = make_ulonglong2(ha.ll, hb.ll);
+            *reinterpret_cast<ulonglong2 *>(Y + sub1) = make_ulonglong2(ha.lh, hb.lh);
+            *reinterpret_cast<ulonglong2 *>(Y + 2 * sub1) = make_ulonglong2(ha.hl, hb.hl);
+            *reinterpret_cast<ulonglong2 *>(Y + 3 * sub1) = make_ulonglong2(ha.hh, hb.hh);
+        }
+        return;
+    }
+    // general path: one 2x2 block per work item, scalar loads
+    const int W1 = g.Wl[1];
+    for (int e = threadIdx.x; e < g.NPP * g.npatch; e += blockDim.x) {
+        const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
+        const int i = fdiv(r, g.d_prow), j = r - i * W1;
         const int b = bg * g.NPP + slot, y = 2 * i, xx = 2 * j;
         const bool x1 = xx + 1 < W, y1 = y + 1 < H;
         float aA = 0.f, bA = 0.f, cA_ = 0.f, dA = 0.f, aB = 0.f, bB = 0.f, cB_ = 0.f, dB = 0.f;
@@ -185,14 +290,14 @@ __device__ __forceinline__ void stage_level1(u64 *sm, const Geom &g, const int *
             }
         }
         u64 *S = sm + (size_t)slot * g.slot_stride;
-        u64 *X = S + off[0] + (y + 2) * p0 + xx + 2;
+        u64 *X = S + off[0] + (y + 2) * p0 + phys_col(xx + 2, h0);  // xx even: xx+2, xx+3 share a chunk
         const u64 a = pk(aA, aB), bq = pk(bA, bB), c = pk(cA_, cB_), d = pk(dA, dB);
         X[0] = a;
         if (x1) X[1] = bq;
         if (y1) X[p0] = c;
         if (x1 && y1) X[p0 + 1] = d;
         const Haar4x2 h = haar2(a, bq, c, d);
-        u64 *Y = S + off[1] + (i + 2) * p1 + j + 2;
+        u64 *Y = S + off[1] + (i + 2) * p1 + phys_col(j + 2, h1);
         Y[0] = h.ll;
         Y[sub1] = h.lh;
         Y[2 * sub1] = h.hl;
@@ -203,14 +308,16 @@ __device__ __forceinline__ void stage_level1(u64 *sm, const Geom &g, const int *
 // Level l >= 2 from the raw LL band of level l-1 (already in shared memory).  Reads one element past
 // an odd grid land in the zero padding.
 __device__ __forceinline__ void stage_level(u64 *sm, const Geom &g, const int *off, int l) {
-    const int Hl = g.Hl[l], Wl = g.Wl[l], n = Hl * Wl;
-    const int pp = g.pitch[l - 1], pl = g.pitch[l], subl = g.rows[l] * pl;
+    const int Wl = g.Wl[l], n = (int)g.d_lvl[l].d;
+    const int pp = g.pitch[l - 1], hp = pp >> 1, pl = g.pitch[l], hl = pl >> 1, subl = g.rows[l] * pl;
     for (int e = threadIdx.x; e < g.NPP * n; e += blockDim.x) {
-        const int slot = e / n, r = e - slot * n, i = r / Wl, j = r - i * Wl;
+        const int slot = fdiv(e, g.d_lvl[l]), r = e - slot * n, i = fdiv(r, g.d_lvlw[l]), j = r - i * Wl;
         u64 *S = sm + (size_t)slot * g.slot_stride;
-        const u64 *src = S + off[l - 1] + (2 * i + 2) * pp + 2 * j + 2;
-        const Haar4x2 h = haar2(src[0], src[1], src[pp], src[pp + 1]);
-        u64 *Y = S + off[l] + (i + 2) * pl + j + 2;
+        const u64 *src = S + off[l - 1] + (2 * i + 2) * pp + phys_col(2 * j + 2, hp);  // even column: one chunk
+        const ulonglong2 top = *reinterpret_cast<const ulonglong2 *>(src);
+        const ulonglong2 bot = *reinterpret_cast<const ulonglong2 *>(src + pp);
+        const Haar4x2 h = haar2(top.x, top.y, bot.x, bot.y);
+        u64 *Y = S + off[l] + (i + 2) * pl + phys_col(j + 2, hl);
         Y[0] = h.ll;
         Y[subl] = h.lh;
         Y[2 * subl] = h.hl;
@@ -218,17 +325,23 @@ __device__ __forceinline__ void stage_level(u64 *sm, const Geom &g, const int *o
     }
 }
 
-// 4x4 output tile of a 5x5 correlation.  `src` points at the window's top-left element (the array's
-// halo of 2 makes window row rr = output row + tap row), 16-byte aligned; w[25] packed weights.
-__device__ __forceinline__ void conv_tile(const u64 *__restrict__ src, int pitch, const u64 *w, u64 (&acc)[4][4]) {
+// 4x4 output tile of a 5x5 correlation.  `src` = array + (4*ty)*pitch + 2*tx points at the even-half
+// word of the window's first chunk (the array's halo of 2 makes window row rr = output row + tap row);
+// the window's four chunks per row are src[0..1], src[half..], src[2..3], src[half+2..].
+__device__ __forceinline__ void conv_tile(const u64 *__restrict__ src, int pitch, const u64 (&w)[KK],
+                                          u64 (&acc)[4][4]) {
+    const int half = pitch >> 1;
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[r][c] = 0ull;
 #pragma unroll
     for (int rr = 0; rr < 8; ++rr) {
-        const ulonglong2 *rp = reinterpret_cast<const ulonglong2 *>(src + rr * pitch);
-        const ulonglong2 q0 = rp[0], q1 = rp[1], q2 = rp[2], q3 = rp[3];
+        const u64 *rp = src + rr * pitch;
+        const ulonglong2 q0 = *reinterpret_cast<const ulonglong2 *>(rp);
+        const ulonglong2 q1 = *reinterpret_cast<const ulonglong2 *>(rp + half);
+        const ulonglong2 q2 = *reinterpret_cast<const ulonglong2 *>(rp + 2);
+        const ulonglong2 q3 = *reinterpret_cast<const ulonglong2 *>(rp + half + 2);
         const u64 in[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
 #pragma unroll
         for (int u = 0; u < 5; ++u) {
@@ -248,10 +361,9 @@ __device__ __forceinline__ void decode_level_item(const Geom &g, int r, int &l, 
     l = 1;
     while (r >= g.lvl_start[l + 1]) ++l;
     r -= g.lvl_start[l];
-    const int nt = g.tx[l] * g.ty[l];
-    sub = r / nt;
-    r -= sub * nt;
-    tyy = r / g.tx[l];
+    sub = fdiv(r, g.d_nt[l]);
+    r -= sub * (int)g.d_nt[l].d;
+    tyy = fdiv(r, g.d_tx[l]);
     txx = r - tyy * g.tx[l];
 }
 
@@ -261,7 +373,7 @@ __device__ __forceinline__ void store_row4(T *__restrict__ p, int x0, int W, boo
 template <>
 __device__ __forceinline__ void store_row4<float>(float *__restrict__ p, int x0, int W, bool vec, float v0, float v1,
                                                   float v2, float v3) {
-    if (vec && x0 + 3 < W) {
+    if (vec) {
         *reinterpret_cast<float4 *>(p) = make_float4(v0, v1, v2, v3);
     } else {
         if (x0 < W) p[0] = v0;
@@ -273,7 +385,7 @@ __device__ __forceinline__ void store_row4<float>(float *__restrict__ p, int x0,
 template <>
 __device__ __forceinline__ void store_row4<__half>(__half *__restrict__ p, int x0, int W, bool vec, float v0, float v1,
                                                    float v2, float v3) {
-    if (vec && x0 + 3 < W) {
+    if (vec) {
         __half2 a = __floats2half2_rn(v0, v1), b = __floats2half2_rn(v2, v3);
         uint2 q;
         q.x = *reinterpret_cast<unsigned *>(&a);
@@ -289,7 +401,7 @@ __device__ __forceinline__ void store_row4<__half>(__half *__restrict__ p, int x
 template <>
 __device__ __forceinline__ void store_row4<__nv_bfloat16>(__nv_bfloat16 *__restrict__ p, int x0, int W, bool vec,
                                                           float v0, float v1, float v2, float v3) {
-    if (vec && x0 + 3 < W) {
+    if (vec) {
         __nv_bfloat162 a = __floats2bfloat162_rn(v0, v1), b = __floats2bfloat162_rn(v2, v3);
         uint2 q;
         q.x = *reinterpret_cast<unsigned *>(&a);
@@ -308,25 +420,39 @@ __device__ __forceinline__ void store_row4<__nv_bfloat16>(__nv_bfloat16 *__restr
 // by 180 degrees and no bias gives grad_x.
 template <typename T, bool FLIP>
 __global__ void __launch_bounds__(MAX_THREADS, 1)
-plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0, const float *__restrict__ s0,
-                 const float *__restrict__ b0, const float *__restrict__ wl, const float *__restrict__ sl,
-                 T *__restrict__ out) {
+plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0,
+                 const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
+                 const float *__restrict__ sl, T *__restrict__ out) {
     extern __shared__ __align__(16) u64 sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
     for (int i = tid; i < g.smem_u64; i += nthr) sm[i] = 0ull;
     u64 *wtab = sm + g.wtab_off;
     const int L = g.L, nlv = g.lvl_start[L + 1];
-    const bool vec = (g.W & 3) == 0;
     const size_t HW = (size_t)g.H * g.W;
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
+    // this thread's base tile never changes: decode it once
+    const int bi = nthr - 1 - tid;
+    const bool has_base = bi < g.NPP * g.nbase;
+    int bslot = 0, tyy = 0, txx = 0;
+    if (has_base) {
+        bslot = fdiv(bi, g.d_nbase);
+        const int r = bi - bslot * g.nbase;
+        tyy = fdiv(r, g.d_tx[0]);
+        txx = r - tyy * g.tx[0];
+    }
+    const u64 *base_src = sm + (size_t)bslot * g.slot_stride + g.offA[0] + 4 * tyy * g.pitch[0] + 2 * txx;
+    int cp_prev = -1;
     __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
         const int cp = u / g.bgroups, bg = u - cp * g.bgroups;
         const int cA = 2 * cp;
         const bool hasB = cA + 1 < g.C;
-        build_weight_table<T>(wtab, g, cA, hasB, FLIP, w0, s0, FLIP ? nullptr : b0, wl, sl);
-        stage_level1<T>(sm, g, g.offA, x, cA, hasB, bg);
+        if (cp != cp_prev) {  // units are channel-pair major: the table survives all images of a pair
+            build_weight_table(wtab, g, cA, hasB, FLIP, w0, s0, FLIP ? nullptr : b0, wl, sl);
+            cp_prev = cp;
+        }
+        stage_input<T>(sm, g, g.offA, x, cA, hasB, bg);
         __syncthreads();
         for (int l = 2; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
@@ -334,50 +460,40 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         }
         // ---- level tiles: Z^l = Wfold^l (*) Y^l
         for (int it = tid; it < g.NPP * nlv; it += nthr) {
-            const int slot = it / nlv;
-            int l, sub, tyy, txx;
-            decode_level_item(g, it - slot * nlv, l, sub, tyy, txx);
-            const u64 *S = sm + (size_t)slot * g.slot_stride;
+            const int slot = fdiv(it, g.d_nlv);
+            int l, sub, ty2, tx2;
+            decode_level_item(g, it - slot * nlv, l, sub, ty2, tx2);
+            u64 *S = sm + (size_t)slot * g.slot_stride;
             const int pl = g.pitch[l];
-            const u64 *src = S + g.offA[l] + sub * g.rows[l] * pl + 4 * tyy * pl + 4 * txx;
             u64 w[KK];
-            const u64 *wt = wtab + (1 + (l - 1) * 4 + sub) * KK;
-#pragma unroll
-            for (int t = 0; t < KK; ++t) w[t] = wt[t];
+            load_weights(wtab + (1 + (l - 1) * 4 + sub) * WT_STRIDE, w);
             u64 acc[4][4];
-            conv_tile(src, pl, w, acc);
+            conv_tile(S + g.offA[l] + sub * g.rows[l] * pl + 4 * ty2 * pl + 2 * tx2, pl, w, acc);
             const int zp = g.zpitch[l];
-            u64 *z = sm + (size_t)slot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + 4 * tyy * zp + 4 * txx;
+            u64 *z = S + g.offZ[l] + sub * g.zrows[l] * zp + 4 * ty2 * zp + 4 * tx2;
+            const int zr_left = g.zrows[l] - 4 * ty2;
+            const bool c0 = 4 * tx2 < zp, c1 = 4 * tx2 + 2 < zp;
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
-                if (4 * tyy + r < g.zrows[l]) {
+                if (r < zr_left) {
                     ulonglong2 *zr = reinterpret_cast<ulonglong2 *>(z + r * zp);
-                    if (4 * txx < zp) zr[0] = make_ulonglong2(acc[r][0], acc[r][1]);
-                    if (4 * txx + 2 < zp) zr[1] = make_ulonglong2(acc[r][2], acc[r][3]);
+                    if (c0) zr[0] = make_ulonglong2(acc[r][0], acc[r][1]);
+                    if (c1) zr[1] = make_ulonglong2(acc[r][2], acc[r][3]);
                 }
             }
         }
         // ---- base tile (at most one per thread), kept in registers across the barrier
-        const int bi = nthr - 1 - tid;
-        const bool has_base = bi < g.NPP * g.nbase;
         u64 acc[4][4];
-        int slot = 0, tyy = 0, txx = 0;
         u64 bias2 = 0ull;
         if (has_base) {
-            slot = bi / g.nbase;
-            const int r = bi - slot * g.nbase;
-            tyy = r / g.tx[0];
-            txx = r - tyy * g.tx[0];
-            const u64 *src = sm + (size_t)slot * g.slot_stride + g.offA[0] + 4 * tyy * g.pitch[0] + 4 * txx;
             u64 w[KK];
-#pragma unroll
-            for (int t = 0; t < KK; ++t) w[t] = wtab[t];
-            conv_tile(src, g.pitch[0], w, acc);
-            bias2 = wtab[(1 + 4 * L) * KK];
+            load_weights(wtab, w);
+            conv_tile(base_src, g.pitch[0], w, acc);
+            bias2 = wtab[KK];
         }
         __syncthreads();
         if (has_base) {
-            const u64 *S = sm + (size_t)slot * g.slot_stride;
+            const u64 *S = sm + (size_t)bslot * g.slot_stride;
             // Proposition 2, level 1: coefficient (2ty+ci, 2tx+cj) feeds pixels (2ci+by, 2cj+bx) of the tile
             if (L >= 1) {
                 const u64 half = pk(0.5f, 0.5f);
@@ -435,27 +551,26 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
                     for (int c = 0; c < 4; ++c) acc[r][c] = add2(acc[r][c], bias2);
             }
-            const int b = bg * g.NPP + slot;
+            const int b = bg * g.NPP + bslot;
             if (b < g.B) {
-                T *oa = out + ((size_t)b * g.C + cA) * HW;
+                T *oa = out + ((size_t)b * g.C + cA) * HW + (size_t)(4 * tyy) * g.W + 4 * txx;
+                const bool vec = g.vec && (4 * txx + 3 < g.W);
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
-                    const int y = 4 * tyy + r;
-                    if (y < g.H) {
+                    if (4 * tyy + r < g.H) {
                         float a0, a1, a2, a3, b0_, b1, b2, b3;
                         upk(acc[r][0], a0, b0_);
                         upk(acc[r][1], a1, b1);
                         upk(acc[r][2], a2, b2);
                         upk(acc[r][3], a3, b3);
-                        T *pa = oa + (size_t)y * g.W + 4 * txx;
-                        store_row4<T>(pa, 4 * txx, g.W, vec, a0, a1, a2, a3);
-                        if (hasB) store_row4<T>(pa + HW, 4 * txx, g.W, vec, b0_, b1, b2, b3);
+                        store_row4<T>(oa + (size_t)r * g.W, 4 * txx, g.W, vec, a0, a1, a2, a3);
+                        if (hasB) store_row4<T>(oa + HW + (size_t)r * g.W, 4 * txx, g.W, vec, b0_, b1, b2, b3);
                     }
                 }
             }
         }
-        // The next unit's staging overwrites x / Y (last read before the barrier above) and the weight
-        // table (bias already copied to a register); Z is next written after the staging barriers.
+        // The next unit's staging overwrites x / Y (last read before the barrier above) and possibly the
+        // weight table (bias already copied to a register); Z is next written after the staging barriers.
     }
 }
 
@@ -465,8 +580,8 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 // units of a channel pair and are flushed to `part0` / `partl` when the pair changes.
 template <typename T>
 __global__ void __launch_bounds__(MAX_THREADS, 1)
-plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go, float *__restrict__ part0,
-                   float *__restrict__ partl /* levels concatenated: level l at l*C*np*100 */) {
+plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
+                   float *__restrict__ part0, float *__restrict__ partl /* level l at l*C*np*100 */) {
     extern __shared__ __align__(16) u64 sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
     for (int i = tid; i < g.smem_u64; i += nthr) sm[i] = 0ull;
@@ -477,6 +592,8 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     const int lvl = active ? (cls == 0 ? 0 : 1 + ((cls - 1) >> 2)) : 0, sub = (cls - 1) & 3;
     const int kth = active ? tid - g.thr_start[cls] : 0, nth = active ? g.thr_start[cls + 1] - g.thr_start[cls] : 1;
     const int ntile = g.tx[lvl] * g.ty[lvl];
+    const int pl = g.pitch[lvl], hl = pl >> 1;
+    const int suboff = (lvl == 0 ? 0 : sub * g.rows[lvl] * pl);
     u64 acc[KK], gsum = 0ull;
 #pragma unroll
     for (int t = 0; t < KK; ++t) acc[t] = 0ull;
@@ -487,8 +604,8 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
         const int cp = u / g.bgroups, bg = u - cp * g.bgroups;
         const int cA = 2 * cp;
         const bool hasB = cA + 1 < g.C;
-        stage_level1<T>(sm, g, g.offA, x, cA, hasB, bg);
-        stage_level1<T>(sm, g, g.offG, go, cA, hasB, bg);
+        stage_input<T>(sm, g, g.offA, x, cA, hasB, bg);
+        stage_input<T>(sm, g, g.offG, go, cA, hasB, bg);
         __syncthreads();
         for (int l = 2; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
@@ -496,19 +613,18 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             __syncthreads();
         }
         if (active) {
-            const int pl = g.pitch[lvl];
-            const int suboff = (lvl == 0 ? 0 : sub * g.rows[lvl] * pl);
             for (int it = kth; it < g.NPP * ntile; it += nth) {
-                const int slot = it / ntile, r = it - slot * ntile;
-                const int tyy = r / g.tx[lvl], txx = r - tyy * g.tx[lvl];
+                const int slot = fdiv(it, g.d_nt[lvl]), r = it - slot * ntile;
+                const int tyy = fdiv(r, g.d_tx[lvl]), txx = r - tyy * g.tx[lvl];
                 const u64 *S = sm + (size_t)slot * g.slot_stride;
-                const u64 *ysrc = S + g.offA[lvl] + suboff + 4 * tyy * pl + 4 * txx;
-                const u64 *dsrc = S + g.offG[lvl] + suboff + (4 * tyy + 2) * pl + 4 * txx + 2;
+                const u64 *ysrc = S + g.offA[lvl] + suboff + 4 * tyy * pl + 2 * txx;
+                // D tile = columns 4tx+2..4tx+5 of rows 4ty+2..: chunk 2tx+1 (odd half) and chunk 2tx+2 (even half)
+                const u64 *dsrc = S + g.offG[lvl] + suboff + (4 * tyy + 2) * pl + 2 * txx;
                 u64 d[4][4];
 #pragma unroll
                 for (int rr = 0; rr < 4; ++rr) {
-                    const ulonglong2 *dp = reinterpret_cast<const ulonglong2 *>(dsrc + rr * pl);
-                    const ulonglong2 q0 = dp[0], q1 = dp[1];
+                    const ulonglong2 q0 = *reinterpret_cast<const ulonglong2 *>(dsrc + rr * pl + hl);
+                    const ulonglong2 q1 = *reinterpret_cast<const ulonglong2 *>(dsrc + rr * pl + 2);
                     d[rr][0] = q0.x; d[rr][1] = q0.y; d[rr][2] = q1.x; d[rr][3] = q1.y;
                 }
                 if (cls == 0) {
@@ -519,8 +635,11 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
                 }
 #pragma unroll
                 for (int rr = 0; rr < 8; ++rr) {
-                    const ulonglong2 *rp = reinterpret_cast<const ulonglong2 *>(ysrc + rr * pl);
-                    const ulonglong2 q0 = rp[0], q1 = rp[1], q2 = rp[2], q3 = rp[3];
+                    const u64 *rp = ysrc + rr * pl;
+                    const ulonglong2 q0 = *reinterpret_cast<const ulonglong2 *>(rp);
+                    const ulonglong2 q1 = *reinterpret_cast<const ulonglong2 *>(rp + hl);
+                    const ulonglong2 q2 = *reinterpret_cast<const ulonglong2 *>(rp + 2);
+                    const ulonglong2 q3 = *reinterpret_cast<const ulonglong2 *>(rp + hl + 2);
                     const u64 in[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
 #pragma unroll
                     for (int uu = 0; uu < 5; ++uu) {
@@ -588,6 +707,25 @@ inline void fill_common(Geom &g, int B, int C, int H, int W, int L) {
     g.lvl_start[0] = 0; g.lvl_start[1] = 0;
     for (int l = 1; l <= L; ++l) g.lvl_start[l + 1] = g.lvl_start[l] + 4 * g.tx[l] * g.ty[l];
     g.ncp = (C + 1) / 2;
+    g.vec = (L >= 1 && (W & 3) == 0) ? 1 : 0;
+    if (L >= 1) {
+        const int prow = g.vec ? W / 4 : g.Wl[1];
+        g.npatch = g.Hl[1] * prow;
+        g.d_npatch = make_fastdiv(g.npatch);
+        g.d_prow = make_fastdiv(prow);
+    } else {
+        g.npatch = H * W;
+        g.d_npatch = make_fastdiv(g.npatch);
+        g.d_prow = make_fastdiv(W);
+    }
+    for (int l = 0; l <= L; ++l) {
+        g.d_lvl[l] = make_fastdiv(g.Hl[l] * g.Wl[l]);
+        g.d_lvlw[l] = make_fastdiv(g.Wl[l]);
+        g.d_nt[l] = make_fastdiv(g.tx[l] * g.ty[l]);
+        g.d_tx[l] = make_fastdiv(g.tx[l]);
+    }
+    g.d_nlv = make_fastdiv(g.lvl_start[L + 1]);
+    g.d_nbase = make_fastdiv(g.nbase);
 }
 
 // Slot layout; returns float2 count per slot.  with_g: second copy of the input pyramid (grad_out);
@@ -619,7 +757,7 @@ inline bool plan_forward(int B, int C, int H, int W, int L, Geom &best, unsigned
     fill_common(g, B, C, H, W, L);
     const int slot = layout_slot(g, false, true);
     const int M = g.lvl_start[L + 1] + g.nbase;
-    const int wtab = (1 + 4 * L) * KK + 1;
+    const int wtab = (1 + 4 * L) * WT_STRIDE;
     bool found = false;
     best.score = -1.0;
     for (int npp = 1; npp <= 64; ++npp) {
