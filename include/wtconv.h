@@ -73,13 +73,15 @@ typedef enum {
 /* desc->flags */
 #define WTCONV_FLAG_TILED_ONLY 1u /* never take the plane-resident kernels (used to test the tiled path) */
 /* Launch-plan overrides for the plane-resident kernels, for tuning experiments (0 = let the planner choose):
- *   bits  8-13  threads per block / 32 of the forward / input-gradient kernel
- *   bits 14-15  blocks per SM of that kernel
- *   bits 16-22  plane pairs per work unit of that kernel
- *   bits 23-29  plane pairs per work unit of the weight-gradient kernel
+ *   bits  8-12  threads per block / 32 of the forward / input-gradient kernel
+ *   bits 13-15  resident blocks per SM of that kernel
+ *   bits 16-21  planes per work unit of that kernel
+ *   bits 22-27  planes per work unit of the weight-gradient kernel
+ *   bits 28-30  resident blocks per SM of the weight-gradient kernel
  * An override that cannot be met (shared memory, registers) makes the call fail with WTCONV_ERR_CUDA. */
-#define WTCONV_TUNE(threads, blocks_per_sm, pairs, wgrad_pairs) \
-    ((((uint32_t)(threads) / 32u) << 8) | ((uint32_t)(blocks_per_sm) << 14) | ((uint32_t)(pairs) << 16) | ((uint32_t)(wgrad_pairs) << 23))
+#define WTCONV_TUNE(threads, blocks_per_sm, planes, wgrad_planes, wgrad_blocks_per_sm)                    \
+    ((((uint32_t)(threads) / 32u) << 8) | ((uint32_t)(blocks_per_sm) << 13) | ((uint32_t)(planes) << 16) | \
+     ((uint32_t)(wgrad_planes) << 22) | ((uint32_t)(wgrad_blocks_per_sm) << 28))
 
 typedef struct {
     int32_t B, C, H, W; /* activation shape */

@@ -2,23 +2,22 @@
 // in shared memory, so the only HBM traffic is the compulsory one (read x, write out).
 //
 // Design
-//  * A block works on PAIRS of planes (channels 2cp and 2cp+1 of the same image).  Every shared
-//    array holds float2 {plane A, plane B} per element and every multiply-add is a packed
-//    fma.rn.f32x2 whose weight operand is {w_A, w_B}: the FP32 pipe takes two FMAs per issued
-//    instruction, which leaves issue slots for the shared-memory loads.
-//  * Per work unit (a channel pair and a group of NPP images): stage x into a zero-haloed array
-//    and run the Haar butterfly of Eq. 5 on chip (Sec. 4.1), level by level from the raw LL band;
-//    then every thread convolves 4x4 output tiles straight out of shared memory with weights that
-//    already carry the scale (Eq. 8); a thread keeps its base-conv tile in registers across one
-//    barrier and then adds the bit-indexed closed-form synthesis of Proposition 2 (Sec. 4.2)
-//    before the only global store.
-//  * Backward = two kernels.  grad_x is the same kernel run on grad_out with the kernels rotated
-//    by 180 degrees (Sec. 2.2: the adjoint of analysis is synthesis and vice versa, so the adjoint
-//    of the whole operator has the operator's own structure).  The weight-gradient kernel stages
-//    the decompositions of x and grad_out and correlates them tile by tile; each thread only ever
-//    works on one (level, subband) class, so its 25 packed accumulators stay in registers across
-//    all images of a channel pair and are reduced once (block tree through shared memory, then
-//    fixed-order fp64 in the epilogue).
+//  * A block works on units of NPL planes of one channel (images b0..b0+NPL-1).  A plane's footprint
+//    (x with a zero halo, the four Haar subbands of every level with halos, the conv outputs Z^l) is
+//    about 58 KB for 56x56, so three to four blocks are resident per SM: while one block is in a
+//    latency-bound phase (staging, synthesis, stores) the others keep the FP32 pipe busy.
+//  * Per unit: stage x into the haloed array and run the Haar butterfly of Eq. 5 on chip (Sec. 4.1),
+//    level by level from the raw LL band; then every thread convolves 4-column x 8-row register tiles
+//    straight out of shared memory (two aligned 16-byte loads per window row, lanes 16 bytes apart: no
+//    bank conflicts) with weights that already carry the scale (Eq. 8).  Level tiles and base tiles are
+//    one item list and one code path; a thread keeps its base tile in registers across one barrier and
+//    then adds the bit-indexed closed-form synthesis of Proposition 2 (Sec. 4.2) before the only store.
+//  * Backward = two kernels.  grad_x is the same kernel run on grad_out with the kernels rotated by 180
+//    degrees (Sec. 2.2: the adjoint of analysis is synthesis and vice versa, so the adjoint of the whole
+//    operator has the operator's own structure).  The weight-gradient kernel stages the decompositions
+//    of x and grad_out and correlates them tile by tile; each thread only ever works on one (level,
+//    subband) class, so its 25 accumulators stay in registers across all images of a channel and are
+//    reduced once (block tree through shared memory, then fixed-order fp64 in the epilogue).
 #pragma once
 #include "common.cuh"
 #include "tiled_kernels.cuh"
@@ -26,58 +25,56 @@
 namespace wt {
 namespace plane {
 
-typedef unsigned long long u64;
 constexpr int MAXL = 8;
 constexpr int KK = 25;
-constexpr int MAX_THREADS = 512;
+constexpr int TH = 8;                        // register tile: 4 columns x TH rows
+constexpr int MAX_THREADS = 256;
 constexpr int NUM_SMS = 148;                 // planning constant (B200); plans must not depend on the device
 constexpr int SMEM_LIMIT = 227 * 1024;       // opt-in dynamic shared memory per block
 constexpr int SMEM_PER_SM = 228 * 1024;      // per SM, 1 KB reserved per resident block
+constexpr int WT_STRIDE = 28;                // floats per class in the weight table (25 taps, 16-byte padded)
+constexpr unsigned WAIT_LIMIT = 1u << 24;    // bounded spin on the copy barrier (never an endless loop)
 
-// ------------------------------------------------------------------ packed fp32x2 helpers
-__device__ __forceinline__ u64 pk(float lo, float hi) {
-    u64 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
+// ------------------------------------------------------------------ bulk-copy (TMA, untiled) helpers
+__device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
-__device__ __forceinline__ void upk(u64 v, float &lo, float &hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long *bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
-    u64 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
+// global -> shared, 16-byte aligned both sides, size a multiple of 16; completion counted on `bar`
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
 }
-__device__ __forceinline__ u64 add2(u64 a, u64 b) {
-    u64 d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
+// Bounded wait for phase `parity` of `bar`; false if it did not complete within WAIT_LIMIT polls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
+    const unsigned a = smem_addr(bar);
+    for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
+        unsigned ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok)
+                     : "r"(a), "r"(parity)
+                     : "memory");
+        if (ok) return true;
+    }
+    return false;
 }
-__device__ __forceinline__ u64 sub2(u64 a, u64 b) {
-    u64 d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ u64 mul2(u64 a, u64 b) {
-    u64 d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
+// order earlier generic-proxy accesses of shared memory before later async-proxy (bulk copy) writes
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Packed Eq. 5 on {A,B} pairs.
-struct Haar4x2 {
-    u64 ll, lh, hl, hh;
-};
-__device__ __forceinline__ Haar4x2 haar2(u64 a, u64 b, u64 c, u64 d) {
-    const u64 half = pk(0.5f, 0.5f);
-    u64 s0 = add2(a, b), s1 = add2(c, d), d0 = sub2(a, b), d1 = sub2(c, d);
-    Haar4x2 r;
-    r.ll = mul2(half, add2(s0, s1));
-    r.lh = mul2(half, sub2(s0, s1));
-    r.hl = mul2(half, add2(d0, d1));
-    r.hh = mul2(half, sub2(d0, d1));
-    return r;
-}
+#ifdef WT_PHASE_TIMING
+__device__ unsigned long long wt_phase_cycles[32];
+#define WT_TICK(i) do { if (threadIdx.x == 0 || threadIdx.x == blockDim.x - 1) { long long now_ = clock64(); atomicAdd(&wt_phase_cycles[(i) + (threadIdx.x ? 16 : 0)], (unsigned long long)(now_ - tick_)); tick_ = now_; } } while (0)
+#define WT_TICK_INIT long long tick_ = clock64();
+#else
+#define WT_TICK(i)
+#define WT_TICK_INIT
+#endif
 
 // ------------------------------------------------------------------ geometry (host-planned, passed by value)
 // Division by a launch-invariant divisor as multiply-high: exact while dividend * divisor < 2^32.
@@ -95,25 +92,30 @@ __device__ __forceinline__ int fdiv(int e, const FastDiv &f) { return f.d == 1 ?
 struct Geom {
     int B, C, H, W, L;
     int Hl[MAXL + 1], Wl[MAXL + 1];        // level grids, index 0 = input
-    int rows[MAXL + 1], pitch[MAXL + 1];   // haloed arrays: pad4(Hl)+4 rows, pitch pad4(Wl)+4 (units of float2)
+    int rows[MAXL + 1], pitch[MAXL + 1];   // haloed arrays: ty*TH+4 rows, pitch pad4(Wl)+4 floats; element (y,x) at (y+2, x+2)
     int offA[MAXL + 1];                    // slot-relative offset of x (l=0) / Y^l subband 0 (subband stride rows*pitch)
     int offG[MAXL + 1];                    // same for grad_out / D^l (weight-gradient kernel only)
     int zrows[MAXL + 1], zpitch[MAXL + 1]; // conv outputs Z^l (forward kernel only)
     int offZ[MAXL + 1];
-    int slot_stride;                       // float2 per plane-pair slot
-    int NPP;                               // plane-pair slots per work unit
-    int tx[MAXL + 1], ty[MAXL + 1];        // 4x4 tiles per level grid (index 0 = base)
-    int lvl_start[MAXL + 2];               // per pair: first level-item of level l (1..L); [L+1] = count
-    int nbase;                             // base tiles per pair
-    int wtab_off;                          // offset of the folded weight table [(1+4L)][26] float2 (+ bias entry)
-    int smem_u64;                          // shared memory in float2 units
-    int bgroups, ncp, units;               // work units = ncp channel pairs x bgroups image groups
+    int slot_stride;                       // floats per plane slot
+    int NPL;                               // plane slots per work unit (images of one channel)
+    int tx[MAXL + 1], ty[MAXL + 1];        // 4 x TH tiles per level grid (index 0 = base)
+    int lvl_start[MAXL + 2];               // per plane: first level-item of level l (1..L); [L+1] = count
+    int nbase;                             // base tiles per plane
+    int wtab_off;                          // offset of the folded weight table [(1+4L)][WT_STRIDE] (bias at [0][25])
+    int smem_floats;
+    int bgroups, units;                    // work units = C channels x bgroups image groups (channel-major)
     int nthreads, nblocks, blocks_per_sm;
-    int vec;                               // 1: W % 4 == 0, rows can be staged with 4-element vector loads
-    int npatch;                            // staging work items per pair (vec: 2x4 pixel patches, else 2x2 blocks)
+    int vec;                               // 1: W % 4 == 0, rows are staged with 4-element vector loads
+    int bulk;                              // 1: planes are fetched one unit ahead with cp.async.bulk into raw_off
+    int raw_off, raw_slot_bytes, plane_bytes;  // raw staging buffer (float offset), bytes per plane slot / per plane
+    int bar_off;                           // float offset of the copy mbarrier (8-byte aligned)
+    int npatch4;                           // 4x4 pixel patches per plane (vec staging of levels 1 and 2 in one pass)
+    FastDiv d_npatch4;
+    int npatch;                            // staging work items per plane (vec: 2x4 pixel patches, else 2x2 blocks)
     FastDiv d_npatch, d_prow;              // / npatch, / (patches per patch-row)
     FastDiv d_lvl[MAXL + 1], d_lvlw[MAXL + 1];  // / (Hl*Wl), / Wl   (levels >= 2 staging)
-    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase;
+    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase, d_bg;
     // weight-gradient kernel: class-major thread allocation and partial-sum slots
     int thr_start[4 * MAXL + 2];
     int np;
@@ -127,197 +129,248 @@ __host__ __device__ inline int block_of_unit(long long v, int nb, int units) {
     return (int)(((v + 1) * nb - 1) / units);
 }
 
-// Shared-memory layout of a haloed array row (pitch float2, pitch % 4 == 0): the 16-byte chunks
-// (two float2) of a row are de-interleaved, even chunks in the first half of the row and odd chunks in
-// the second.  A thread's 4x4 tile window starts at column 4*tx, so lanes of a warp read chunk
-// 2*tx + j: for fixed j consecutive lanes hit consecutive 16-byte words - no bank conflicts.
-__device__ __forceinline__ int phys_col(int col, int half) {
-    return ((col >> 1) & 1) * half + ((col >> 2) << 1) + (col & 1);
-}
-
-constexpr int WT_STRIDE = 26;  // float2 per class in the weight table (25 taps, padded to 16 bytes)
-
 // ------------------------------------------------------------------ shared device pieces
-__device__ __forceinline__ void build_weight_table(u64 *wtab, const Geom &g, int cA, bool hasB, bool flip,
+__device__ __forceinline__ void build_weight_table(float *wtab, const Geom &g, int c, bool flip,
                                                    const float *__restrict__ w0, const float *__restrict__ s0,
                                                    const float *__restrict__ b0, const float *__restrict__ wl,
                                                    const float *__restrict__ sl) {
-    const int ncls = 1 + 4 * g.L, cB = cA + 1;
+    const int ncls = 1 + 4 * g.L;
     for (int e = threadIdx.x; e < ncls * KK; e += blockDim.x) {
         const int cls = e / KK, t = e - cls * KK, src = flip ? (KK - 1 - t) : t;
-        float wa, wb = 0.f;
+        float w;
         if (cls == 0) {
-            wa = __ldg(w0 + cA * KK + src) * __ldg(s0 + cA);
-            if (hasB) wb = __ldg(w0 + cB * KK + src) * __ldg(s0 + cB);
+            w = __ldg(w0 + c * KK + src) * __ldg(s0 + c);
         } else {
             const int l = (cls - 1) >> 2, sub = (cls - 1) & 3;
-            const size_t ia = ((size_t)l * g.C + cA) * 4 + sub, ib = ((size_t)l * g.C + cB) * 4 + sub;
-            wa = __ldg(wl + ia * KK + src) * __ldg(sl + ia);
-            if (hasB) wb = __ldg(wl + ib * KK + src) * __ldg(sl + ib);
+            const size_t i = ((size_t)l * g.C + c) * 4 + sub;
+            w = __ldg(wl + i * KK + src) * __ldg(sl + i);
         }
-        wtab[cls * WT_STRIDE + t] = pk(wa, wb);  // Eq. 8: scale folded into the weight
+        wtab[cls * WT_STRIDE + t] = w;  // Eq. 8: scale folded into the weight
     }
-    if (threadIdx.x == 0) {
-        float ba = 0.f, bb = 0.f;
-        if (b0) {
-            ba = __ldg(s0 + cA) * __ldg(b0 + cA);
-            if (hasB) bb = __ldg(s0 + cB) * __ldg(b0 + cB);
-        }
-        wtab[KK] = pk(ba, bb);  // the spare 26th entry of class 0
-    }
+    if (threadIdx.x == 0) wtab[KK] = b0 ? __ldg(s0 + c) * __ldg(b0 + c) : 0.f;  // spare entry of class 0
 }
 
-__device__ __forceinline__ void load_weights(const u64 *wt, u64 (&w)[KK]) {
-    const ulonglong2 *q = reinterpret_cast<const ulonglong2 *>(wt);
+__device__ __forceinline__ void load_weights(const float *wt, float (&w)[KK]) {
+    const float4 *q = reinterpret_cast<const float4 *>(wt);
 #pragma unroll
-    for (int t = 0; t < 12; ++t) {
-        const ulonglong2 v = q[t];
-        w[2 * t] = v.x;
-        w[2 * t + 1] = v.y;
+    for (int t = 0; t < 6; ++t) {
+        const float4 v = q[t];
+        w[4 * t] = v.x; w[4 * t + 1] = v.y; w[4 * t + 2] = v.z; w[4 * t + 3] = v.w;
     }
     w[24] = wt[24];
 }
 
-template <typename T>
-__device__ __forceinline__ void load4(const T *p, float (&v)[4]);
-template <>
-__device__ __forceinline__ void load4<float>(const float *p, float (&v)[4]) {
+// four consecutive activations (16-byte aligned for float, 8-byte for the 16-bit types)
+__device__ __forceinline__ void load4(const float *p, float (&v)[4]) {
     const float4 q = __ldg(reinterpret_cast<const float4 *>(p));
     v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
 }
-template <>
-__device__ __forceinline__ void load4<__half>(const __half *p, float (&v)[4]) {
+__device__ __forceinline__ void load4(const __half *p, float (&v)[4]) {
     const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
     const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
     const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
     v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
 }
-template <>
-__device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16 *p, float (&v)[4]) {
+__device__ __forceinline__ void load4(const __nv_bfloat16 *p, float (&v)[4]) {
     const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
     const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x));
     const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.y));
     v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
 }
 
-// Stage the planes of one unit: x into the haloed array `off[0]` and its level-1 Haar subbands (Eq. 5)
-// into `off[1]`, both planes of each pair interleaved.  Pixels beyond H x W are never written and stay
-// zero (odd-size padding and conv halo); images beyond the batch are written as zeros.
-template <typename T>
-__device__ __forceinline__ void stage_input(u64 *sm, const Geom &g, const int *off, const T *__restrict__ x, int cA,
-                                            bool hasB, int bg) {
+// the same from shared memory (a raw plane a bulk copy landed there)
+__device__ __forceinline__ void load4s(const float *p, float (&v)[4]) {
+    const float4 q = *reinterpret_cast<const float4 *>(p);
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+}
+__device__ __forceinline__ void load4s(const __half *p, float (&v)[4]) {
+    const uint2 q = *reinterpret_cast<const uint2 *>(p);
+    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+__device__ __forceinline__ void load4s(const __nv_bfloat16 *p, float (&v)[4]) {
+    const uint2 q = *reinterpret_cast<const uint2 *>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.y));
+    v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+}
+__device__ __forceinline__ float ldf_plain(const float *p) { return *p; }
+__device__ __forceinline__ float ldf_plain(const __half *p) { return __half2float(*p); }
+__device__ __forceinline__ float ldf_plain(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+template <typename T, bool RAW>
+__device__ __forceinline__ float ld1(const T *p) { return RAW ? ldf_plain(p) : ldf(p); }
+template <typename T, bool RAW>
+__device__ __forceinline__ void ld4(const T *p, float (&v)[4]) {
+    if (RAW) load4s(p, v); else load4(p, v);
+}
+
+// Stage the planes of one unit (channel c, images bg*NPL ..): x into the haloed array `off[0]`, its
+// level-1 Haar subbands (Eq. 5) into `off[1]` and, on the vector path with L >= 2, the level-2 subbands
+// into `off[2]` in the same pass (returns the first level that still has to be staged).  RAW = true reads
+// plane slot s from the raw shared buffer at src + s * slot_elems (a bulk copy put it there); RAW = false
+// reads global memory.  Pixels beyond H x W are never written and stay zero (odd-size padding and conv
+// halo); images beyond the batch are written as zeros.
+template <typename T, bool RAW>
+__device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *off, const T *__restrict__ src, int c,
+                                           int bg) {
     const int H = g.H, W = g.W;
     const size_t HW = (size_t)H * W;
-    const int p0 = g.pitch[0], h0 = p0 >> 1;
+    const int p0 = g.pitch[0];
+    const size_t slot_elems = RAW ? (size_t)g.raw_slot_bytes / sizeof(T) : 0;
     if (g.L == 0) {
-        for (int e = threadIdx.x; e < g.NPP * H * W; e += blockDim.x) {
-            const int slot = e / (H * W), r = e - slot * (H * W), y = r / W, xx = r - y * W;
-            const int b = bg * g.NPP + slot;
-            float va = 0.f, vb = 0.f;
-            if (b < g.B) {
-                const T *pa = x + ((size_t)b * g.C + cA) * HW + r;
-                va = ldf(pa);
-                if (hasB) vb = ldf(pa + HW);
-            }
-            sm[(size_t)slot * g.slot_stride + off[0] + (y + 2) * p0 + phys_col(xx + 2, h0)] = pk(va, vb);
+        for (int e = threadIdx.x; e < g.NPL * H * W; e += blockDim.x) {
+            const int slot = fdiv(e, g.d_npatch), r = e - slot * (H * W), y = fdiv(r, g.d_prow), xx = r - y * W;
+            const int b = bg * g.NPL + slot;
+            const T *pa = RAW ? src + slot * slot_elems + r : src + ((size_t)b * g.C + c) * HW + r;
+            sm[(size_t)slot * g.slot_stride + off[0] + (y + 2) * p0 + xx + 2] = b < g.B ? ld1<T, RAW>(pa) : 0.f;
         }
-        return;
+        return 1;
     }
-    const int p1 = g.pitch[1], h1 = p1 >> 1, sub1 = g.rows[1] * p1;
-    if (g.vec) {
-        // work item = 2 rows x 4 columns of both planes: two Haar blocks, whole 16-byte chunks everywhere
-        for (int e = threadIdx.x; e < g.NPP * g.npatch; e += blockDim.x) {
-            const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
-            const int i = fdiv(r, g.d_prow), q = r - i * (int)g.d_prow.d;
-            const int b = bg * g.NPP + slot, y = 2 * i;
-            const bool y1 = y + 1 < H;
-            float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f}, b0[4] = {0.f, 0.f, 0.f, 0.f},
-                  b1[4] = {0.f, 0.f, 0.f, 0.f};
+    const int p1 = g.pitch[1], sub1 = g.rows[1] * p1;
+    if (g.vec && g.L >= 2) {
+        // work item = 4 rows x 4 columns: four level-1 blocks and the level-2 block above them
+        const int p2 = g.pitch[2], sub2 = g.rows[2] * p2;
+        for (int e = threadIdx.x; e < g.NPL * g.npatch4; e += blockDim.x) {
+            const int slot = fdiv(e, g.d_npatch4), r = e - slot * g.npatch4;
+            const int i2 = fdiv(r, g.d_prow), q = r - i2 * (int)g.d_prow.d;
+            const int b = bg * g.NPL + slot, y = 4 * i2;
+            float a[4][4];
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) a[rr][cc] = 0.f;
             if (b < g.B) {
-                const T *pa = x + ((size_t)b * g.C + cA) * HW + (size_t)y * W + 4 * q;
-                load4<T>(pa, a0);
-                if (y1) load4<T>(pa + W, a1);
-                if (hasB) {
-                    load4<T>(pa + HW, b0);
-                    if (y1) load4<T>(pa + HW + W, b1);
+                const T *pa = (RAW ? src + slot * slot_elems : src + ((size_t)b * g.C + c) * HW) + (size_t)y * W + 4 * q;
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr)
+                    if (y + rr < H) ld4<T, RAW>(pa + (size_t)rr * W, a[rr]);
+            }
+            float *S = sm + (size_t)slot * g.slot_stride;
+            float *X = S + off[0] + (y + 2) * p0 + 4 * q + 2;  // 8-byte aligned
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+                if (y + rr < H) {
+                    *reinterpret_cast<float2 *>(X + rr * p0) = make_float2(a[rr][0], a[rr][1]);
+                    *reinterpret_cast<float2 *>(X + rr * p0 + 2) = make_float2(a[rr][2], a[rr][3]);
                 }
             }
-            u64 *S = sm + (size_t)slot * g.slot_stride;
-            u64 r0v[4], r1v[4];
+            Haar4 h[2][2];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                r0v[c] = pk(a0[c], b0[c]);
-                r1v[c] = pk(a1[c], b1[c]);
+            for (int bi = 0; bi < 2; ++bi)
+#pragma unroll
+                for (int bj = 0; bj < 2; ++bj)
+                    h[bi][bj] = haar_butterfly(a[2 * bi][2 * bj], a[2 * bi][2 * bj + 1], a[2 * bi + 1][2 * bj],
+                                               a[2 * bi + 1][2 * bj + 1]);
+            float *Y = S + off[1] + (2 * i2 + 2) * p1 + 2 * q + 2;
+#pragma unroll
+            for (int bi = 0; bi < 2; ++bi) {
+                *reinterpret_cast<float2 *>(Y + bi * p1) = make_float2(h[bi][0].ll, h[bi][1].ll);
+                *reinterpret_cast<float2 *>(Y + bi * p1 + sub1) = make_float2(h[bi][0].lh, h[bi][1].lh);
+                *reinterpret_cast<float2 *>(Y + bi * p1 + 2 * sub1) = make_float2(h[bi][0].hl, h[bi][1].hl);
+                *reinterpret_cast<float2 *>(Y + bi * p1 + 3 * sub1) = make_float2(h[bi][0].hh, h[bi][1].hh);
             }
-            // columns 4q+2 .. 4q+5 = chunk 2q+1 (odd half, index q) and chunk 2q+2 (even half, index q+1)
-            u64 *X = S + off[0] + (y + 2) * p0;
-            *reinterpret_cast<ulonglong2 *>(X + h0 + 2 * q) = make_ulonglong2(r0v[0], r0v[1]);
-            *reinterpret_cast<ulonglong2 *>(X + 2 * q + 2) = make_ulonglong2(r0v[2], r0v[3]);
-            if (y1) {
-                *reinterpret_cast<ulonglong2 *>(X + p0 + h0 + 2 * q) = make_ulonglong2(r1v[0], r1v[1]);
-                *reinterpret_cast<ulonglong2 *>(X + p0 + 2 * q + 2) = make_ulonglong2(r1v[2], r1v[3]);
-            }
-            const Haar4x2 ha = haar2(r0v[0], r0v[1], r1v[0], r1v[1]), hb = haar2(r0v[2], r0v[3], r1v[2], r1v[3]);
-            // level-1 columns 2q+2, 2q+3 = chunk q+1
-            u64 *Y = S + off[1] + (i + 2) * p1 + ((q + 1) & 1) * h1 + ((q + 1) >> 1) * 2;
-            *reinterpret_cast<ulonglong2 *>(Y) = make_ulonglong2(ha.ll, hb.ll);
-            *reinterpret_cast<ulonglong2 *>(Y + sub1) = make_ulonglong2(ha.lh, hb.lh);
-            *reinterpret_cast<ulonglong2 *>(Y + 2 * sub1) = make_ulonglong2(ha.hl, hb.hl);
-            *reinterpret_cast<ulonglong2 *>(Y + 3 * sub1) = make_ulonglong2(ha.hh, hb.hh);
+            const Haar4 h2 = haar_butterfly(h[0][0].ll, h[0][1].ll, h[1][0].ll, h[1][1].ll);
+            float *Y2 = S + off[2] + (i2 + 2) * p2 + q + 2;
+            Y2[0] = h2.ll;
+            Y2[sub2] = h2.lh;
+            Y2[2 * sub2] = h2.hl;
+            Y2[3 * sub2] = h2.hh;
         }
-        return;
+        return 3;
+    }
+    if (g.vec) {
+        // work item = 2 rows x 4 columns: two Haar blocks
+        for (int e = threadIdx.x; e < g.NPL * g.npatch; e += blockDim.x) {
+            const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
+            const int i = fdiv(r, g.d_prow), q = r - i * (int)g.d_prow.d;
+            const int b = bg * g.NPL + slot, y = 2 * i;
+            const bool y1 = y + 1 < H;
+            float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+            if (b < g.B) {
+                const T *pa = (RAW ? src + slot * slot_elems : src + ((size_t)b * g.C + c) * HW) + (size_t)y * W + 4 * q;
+                ld4<T, RAW>(pa, a0);
+                if (y1) ld4<T, RAW>(pa + W, a1);
+            }
+            float *S = sm + (size_t)slot * g.slot_stride;
+            float *X = S + off[0] + (y + 2) * p0 + 4 * q + 2;  // 8-byte aligned
+            *reinterpret_cast<float2 *>(X) = make_float2(a0[0], a0[1]);
+            *reinterpret_cast<float2 *>(X + 2) = make_float2(a0[2], a0[3]);
+            if (y1) {
+                *reinterpret_cast<float2 *>(X + p0) = make_float2(a1[0], a1[1]);
+                *reinterpret_cast<float2 *>(X + p0 + 2) = make_float2(a1[2], a1[3]);
+            }
+            const Haar4 ha = haar_butterfly(a0[0], a0[1], a1[0], a1[1]), hb = haar_butterfly(a0[2], a0[3], a1[2], a1[3]);
+            float *Y = S + off[1] + (i + 2) * p1 + 2 * q + 2;
+            *reinterpret_cast<float2 *>(Y) = make_float2(ha.ll, hb.ll);
+            *reinterpret_cast<float2 *>(Y + sub1) = make_float2(ha.lh, hb.lh);
+            *reinterpret_cast<float2 *>(Y + 2 * sub1) = make_float2(ha.hl, hb.hl);
+            *reinterpret_cast<float2 *>(Y + 3 * sub1) = make_float2(ha.hh, hb.hh);
+        }
+        return 2;
     }
     // general path: one 2x2 block per work item, scalar loads
     const int W1 = g.Wl[1];
-    for (int e = threadIdx.x; e < g.NPP * g.npatch; e += blockDim.x) {
+    for (int e = threadIdx.x; e < g.NPL * g.npatch; e += blockDim.x) {
         const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
         const int i = fdiv(r, g.d_prow), j = r - i * W1;
-        const int b = bg * g.NPP + slot, y = 2 * i, xx = 2 * j;
+        const int b = bg * g.NPL + slot, y = 2 * i, xx = 2 * j;
         const bool x1 = xx + 1 < W, y1 = y + 1 < H;
-        float aA = 0.f, bA = 0.f, cA_ = 0.f, dA = 0.f, aB = 0.f, bB = 0.f, cB_ = 0.f, dB = 0.f;
+        float a = 0.f, bq = 0.f, cq = 0.f, d = 0.f;
         if (b < g.B) {
-            const T *pa = x + ((size_t)b * g.C + cA) * HW + (size_t)y * W + xx;
-            aA = ldf(pa);
-            if (x1) bA = ldf(pa + 1);
-            if (y1) cA_ = ldf(pa + W);
-            if (x1 && y1) dA = ldf(pa + W + 1);
-            if (hasB) {
-                const T *pb = pa + HW;
-                aB = ldf(pb);
-                if (x1) bB = ldf(pb + 1);
-                if (y1) cB_ = ldf(pb + W);
-                if (x1 && y1) dB = ldf(pb + W + 1);
-            }
+            const T *pa = (RAW ? src + slot * slot_elems : src + ((size_t)b * g.C + c) * HW) + (size_t)y * W + xx;
+            a = ld1<T, RAW>(pa);
+            if (x1) bq = ld1<T, RAW>(pa + 1);
+            if (y1) cq = ld1<T, RAW>(pa + W);
+            if (x1 && y1) d = ld1<T, RAW>(pa + W + 1);
         }
-        u64 *S = sm + (size_t)slot * g.slot_stride;
-        u64 *X = S + off[0] + (y + 2) * p0 + phys_col(xx + 2, h0);  // xx even: xx+2, xx+3 share a chunk
-        const u64 a = pk(aA, aB), bq = pk(bA, bB), c = pk(cA_, cB_), d = pk(dA, dB);
+        float *S = sm + (size_t)slot * g.slot_stride;
+        float *X = S + off[0] + (y + 2) * p0 + xx + 2;
         X[0] = a;
         if (x1) X[1] = bq;
-        if (y1) X[p0] = c;
+        if (y1) X[p0] = cq;
         if (x1 && y1) X[p0 + 1] = d;
-        const Haar4x2 h = haar2(a, bq, c, d);
-        u64 *Y = S + off[1] + (i + 2) * p1 + phys_col(j + 2, h1);
+        const Haar4 h = haar_butterfly(a, bq, cq, d);
+        float *Y = S + off[1] + (i + 2) * p1 + j + 2;
         Y[0] = h.ll;
         Y[sub1] = h.lh;
         Y[2 * sub1] = h.hl;
         Y[3 * sub1] = h.hh;
     }
+    return 2;
+}
+
+// Issue the bulk copies of one unit's planes into the raw buffer (one thread): plane slot s receives image
+// bg*NPL+s of channel c; slots beyond the batch are skipped.  `extra_bytes` lets a caller that copies a
+// second tensor on the same barrier announce all bytes with one expect_tx.
+template <typename T>
+__device__ __forceinline__ void issue_unit_copies(unsigned long long *bar, char *raw, const Geom &g,
+                                                  const T *__restrict__ src, const T *__restrict__ src2, int c, int bg) {
+    int nvalid = g.B - bg * g.NPL;
+    if (nvalid > g.NPL) nvalid = g.NPL;
+    const unsigned per = (unsigned)g.plane_bytes;
+    mbar_expect_tx(bar, per * nvalid * (src2 ? 2u : 1u));
+    const size_t HW = (size_t)g.H * g.W;
+    for (int s2 = 0; s2 < nvalid; ++s2) {
+        const size_t po = ((size_t)(bg * g.NPL + s2) * g.C + c) * HW;
+        bulk_g2s(raw + (size_t)s2 * g.raw_slot_bytes, src + po, per, bar);
+        if (src2) bulk_g2s(raw + (size_t)(g.NPL + s2) * g.raw_slot_bytes, src2 + po, per, bar);
+    }
 }
 
 // Level l >= 2 from the raw LL band of level l-1 (already in shared memory).  Reads one element past
 // an odd grid land in the zero padding.
-__device__ __forceinline__ void stage_level(u64 *sm, const Geom &g, const int *off, int l) {
+__device__ __forceinline__ void stage_level(float *sm, const Geom &g, const int *off, int l) {
     const int Wl = g.Wl[l], n = (int)g.d_lvl[l].d;
-    const int pp = g.pitch[l - 1], hp = pp >> 1, pl = g.pitch[l], hl = pl >> 1, subl = g.rows[l] * pl;
-    for (int e = threadIdx.x; e < g.NPP * n; e += blockDim.x) {
+    const int pp = g.pitch[l - 1], pl = g.pitch[l], subl = g.rows[l] * pl;
+    for (int e = threadIdx.x; e < g.NPL * n; e += blockDim.x) {
         const int slot = fdiv(e, g.d_lvl[l]), r = e - slot * n, i = fdiv(r, g.d_lvlw[l]), j = r - i * Wl;
-        u64 *S = sm + (size_t)slot * g.slot_stride;
-        const u64 *src = S + off[l - 1] + (2 * i + 2) * pp + phys_col(2 * j + 2, hp);  // even column: one chunk
-        const ulonglong2 top = *reinterpret_cast<const ulonglong2 *>(src);
-        const ulonglong2 bot = *reinterpret_cast<const ulonglong2 *>(src + pp);
-        const Haar4x2 h = haar2(top.x, top.y, bot.x, bot.y);
-        u64 *Y = S + off[l] + (i + 2) * pl + phys_col(j + 2, hl);
+        float *S = sm + (size_t)slot * g.slot_stride;
+        const float *src = S + off[l - 1] + (2 * i + 2) * pp + 2 * j + 2;  // even column: 8-byte aligned
+        const float2 top = *reinterpret_cast<const float2 *>(src);
+        const float2 bot = *reinterpret_cast<const float2 *>(src + pp);
+        const Haar4 h = haar_butterfly(top.x, top.y, bot.x, bot.y);
+        float *Y = S + off[l] + (i + 2) * pl + j + 2;
         Y[0] = h.ll;
         Y[subl] = h.lh;
         Y[2 * subl] = h.hl;
@@ -325,38 +378,34 @@ __device__ __forceinline__ void stage_level(u64 *sm, const Geom &g, const int *o
     }
 }
 
-// 4x4 output tile of a 5x5 correlation.  `src` = array + (4*ty)*pitch + 2*tx points at the even-half
-// word of the window's first chunk (the array's halo of 2 makes window row rr = output row + tap row);
-// the window's four chunks per row are src[0..1], src[half..], src[2..3], src[half+2..].
-__device__ __forceinline__ void conv_tile(const u64 *__restrict__ src, int pitch, const u64 (&w)[KK],
-                                          u64 (&acc)[4][4]) {
-    const int half = pitch >> 1;
+// 4-column x TH-row output tile of a 5x5 correlation.  `src` = array + (TH*ty)*pitch + 4*tx is the
+// window's top-left element (the array's halo of 2 makes window row rr = output row + tap row), 16-byte
+// aligned; eight floats per window row.
+__device__ __forceinline__ void conv_tile(const float *__restrict__ src, int pitch, const float (&w)[KK],
+                                          float (&acc)[TH][4]) {
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
+    for (int r = 0; r < TH; ++r)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) acc[r][c] = 0ull;
+        for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
 #pragma unroll
-    for (int rr = 0; rr < 8; ++rr) {
-        const u64 *rp = src + rr * pitch;
-        const ulonglong2 q0 = *reinterpret_cast<const ulonglong2 *>(rp);
-        const ulonglong2 q1 = *reinterpret_cast<const ulonglong2 *>(rp + half);
-        const ulonglong2 q2 = *reinterpret_cast<const ulonglong2 *>(rp + 2);
-        const ulonglong2 q3 = *reinterpret_cast<const ulonglong2 *>(rp + half + 2);
-        const u64 in[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
+    for (int rr = 0; rr < TH + 4; ++rr) {
+        const float4 q0 = *reinterpret_cast<const float4 *>(src + rr * pitch);
+        const float4 q1 = *reinterpret_cast<const float4 *>(src + rr * pitch + 4);
+        const float in[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
         for (int u = 0; u < 5; ++u) {
             const int r = rr - u;
-            if (r >= 0 && r < 4) {
+            if (r >= 0 && r < TH) {
 #pragma unroll
                 for (int v = 0; v < 5; ++v)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) acc[r][c] = fma2(w[u * 5 + v], in[c + v], acc[r][c]);
+                    for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(w[u * 5 + v], in[c + v], acc[r][c]);
             }
         }
     }
 }
 
-// Decode a level item of one pair: r in [0, lvl_start[L+1]) -> (level, subband, tile row, tile col).
+// Decode a level item of one plane: r in [0, lvl_start[L+1]) -> (level, subband, tile row, tile col).
 __device__ __forceinline__ void decode_level_item(const Geom &g, int r, int &l, int &sub, int &tyy, int &txx) {
     l = 1;
     while (r >= g.lvl_start[l + 1]) ++l;
@@ -367,224 +416,246 @@ __device__ __forceinline__ void decode_level_item(const Geom &g, int r, int &l, 
     txx = r - tyy * g.tx[l];
 }
 
-template <typename T>
-__device__ __forceinline__ void store_row4(T *__restrict__ p, int x0, int W, bool vec, float v0, float v1, float v2,
-                                           float v3);
-template <>
-__device__ __forceinline__ void store_row4<float>(float *__restrict__ p, int x0, int W, bool vec, float v0, float v1,
-                                                  float v2, float v3) {
+__device__ __forceinline__ void store_row4(float *__restrict__ p, int x0, int W, bool vec, const float *v) {
     if (vec) {
-        *reinterpret_cast<float4 *>(p) = make_float4(v0, v1, v2, v3);
+        *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
     } else {
-        if (x0 < W) p[0] = v0;
-        if (x0 + 1 < W) p[1] = v1;
-        if (x0 + 2 < W) p[2] = v2;
-        if (x0 + 3 < W) p[3] = v3;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (x0 + c < W) p[c] = v[c];
     }
 }
-template <>
-__device__ __forceinline__ void store_row4<__half>(__half *__restrict__ p, int x0, int W, bool vec, float v0, float v1,
-                                                   float v2, float v3) {
+__device__ __forceinline__ void store_row4(__half *__restrict__ p, int x0, int W, bool vec, const float *v) {
     if (vec) {
-        __half2 a = __floats2half2_rn(v0, v1), b = __floats2half2_rn(v2, v3);
+        __half2 a = __floats2half2_rn(v[0], v[1]), b = __floats2half2_rn(v[2], v[3]);
         uint2 q;
         q.x = *reinterpret_cast<unsigned *>(&a);
         q.y = *reinterpret_cast<unsigned *>(&b);
         *reinterpret_cast<uint2 *>(p) = q;
     } else {
-        if (x0 < W) p[0] = __float2half_rn(v0);
-        if (x0 + 1 < W) p[1] = __float2half_rn(v1);
-        if (x0 + 2 < W) p[2] = __float2half_rn(v2);
-        if (x0 + 3 < W) p[3] = __float2half_rn(v3);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (x0 + c < W) p[c] = __float2half_rn(v[c]);
     }
 }
-template <>
-__device__ __forceinline__ void store_row4<__nv_bfloat16>(__nv_bfloat16 *__restrict__ p, int x0, int W, bool vec,
-                                                          float v0, float v1, float v2, float v3) {
+__device__ __forceinline__ void store_row4(__nv_bfloat16 *__restrict__ p, int x0, int W, bool vec, const float *v) {
     if (vec) {
-        __nv_bfloat162 a = __floats2bfloat162_rn(v0, v1), b = __floats2bfloat162_rn(v2, v3);
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
         uint2 q;
         q.x = *reinterpret_cast<unsigned *>(&a);
         q.y = *reinterpret_cast<unsigned *>(&b);
         *reinterpret_cast<uint2 *>(p) = q;
     } else {
-        if (x0 < W) p[0] = __float2bfloat16_rn(v0);
-        if (x0 + 1 < W) p[1] = __float2bfloat16_rn(v1);
-        if (x0 + 2 < W) p[2] = __float2bfloat16_rn(v2);
-        if (x0 + 3 < W) p[3] = __float2bfloat16_rn(v3);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (x0 + c < W) p[c] = __float2bfloat16_rn(v[c]);
     }
 }
 
 // ------------------------------------------------------------------ forward / input-gradient kernel
+// Adds the Proposition 2 terms of all levels to one 4x4 pixel block (block row t4, block column tx of
+// the plane) held in a[0..3][0..3]; `bias` is the folded bias.
+__device__ __forceinline__ void synth_block(const float *S, const Geom &g, int t4, int txx, float bias, float (*a)[4]) {
+    const int L = g.L;
+    // level 1: coefficient (2*t4+ci, 2*tx+cj) feeds pixels (2ci+by, 2cj+bx) of the block
+    if (L >= 1) {
+        const int zp = g.zpitch[1], zs = g.zrows[1] * zp;
+        const float *z = S + g.offZ[1] + (2 * t4) * zp + 2 * txx;
+#pragma unroll
+        for (int ci = 0; ci < 2; ++ci) {
+            const float2 ll = *reinterpret_cast<const float2 *>(z + ci * zp);
+            const float2 lh = *reinterpret_cast<const float2 *>(z + zs + ci * zp);
+            const float2 hl = *reinterpret_cast<const float2 *>(z + 2 * zs + ci * zp);
+            const float2 hh = *reinterpret_cast<const float2 *>(z + 3 * zs + ci * zp);
+#pragma unroll
+            for (int cj = 0; cj < 2; ++cj) {
+                const float LLv = cj ? ll.y : ll.x, LHv = cj ? lh.y : lh.x, HLv = cj ? hl.y : hl.x,
+                            HHv = cj ? hh.y : hh.x;
+                const float pp = LLv + LHv, pm = LLv - LHv, qp = HLv + HHv, qm = HLv - HHv;
+                a[2 * ci][2 * cj] = fmaf(0.5f, pp + qp, a[2 * ci][2 * cj]);
+                a[2 * ci][2 * cj + 1] = fmaf(0.5f, pp - qp, a[2 * ci][2 * cj + 1]);
+                a[2 * ci + 1][2 * cj] = fmaf(0.5f, pm + qm, a[2 * ci + 1][2 * cj]);
+                a[2 * ci + 1][2 * cj + 1] = fmaf(0.5f, pm - qm, a[2 * ci + 1][2 * cj + 1]);
+            }
+        }
+    }
+    if (L >= 2) {
+        // levels >= 3: the whole block sits in one quadrant of the coefficient's 2^l x 2^l block
+        float deep = bias, scale = 0.25f;
+        for (int l = 3; l <= L; ++l) {
+            scale *= 0.5f;
+            const int zp = g.zpitch[l], zs = g.zrows[l] * zp;
+            const float *z = S + g.offZ[l] + (t4 >> (l - 2)) * zp + (txx >> (l - 2));
+            const float sy = ((t4 >> (l - 3)) & 1) ? -1.f : 1.f, sx = ((txx >> (l - 3)) & 1) ? -1.f : 1.f;
+            const float p = fmaf(sy, z[zs], z[0]), q = fmaf(sy, z[3 * zs], z[2 * zs]);
+            deep = fmaf(scale, fmaf(sx, q, p), deep);
+        }
+        // level 2: coefficient (t4, tx); pixel (r, c) of the block takes its signs from (r>>1, c>>1)
+        const int zp = g.zpitch[2], zs = g.zrows[2] * zp;
+        const float *z = S + g.offZ[2] + t4 * zp + txx;
+        const float LLv = z[0], LHv = z[zs], HLv = z[2 * zs], HHv = z[3 * zs];
+        const float pp = LLv + LHv, pm = LLv - LHv, qp = HLv + HHv, qm = HLv - HHv;
+        float t2[2][2];
+        t2[0][0] = fmaf(0.25f, pp + qp, deep);
+        t2[0][1] = fmaf(0.25f, pp - qp, deep);
+        t2[1][0] = fmaf(0.25f, pm + qm, deep);
+        t2[1][1] = fmaf(0.25f, pm - qm, deep);
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) a[r][c] += t2[r >> 1][c >> 1];
+    } else {
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) a[r][c] += bias;
+    }
+}
+
 // FLIP = false: out = WTConv(x).  FLIP = true: the same dataflow on grad_out with every kernel rotated
-// by 180 degrees and no bias gives grad_x.
-template <typename T, bool FLIP>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
+// by 180 degrees and no bias gives grad_x.  MINB = resident blocks per SM the register budget is sized for.
+template <typename T, bool FLIP, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
 plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0,
                  const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
-                 const float *__restrict__ sl, T *__restrict__ out) {
-    extern __shared__ __align__(16) u64 sm[];
+                 const float *__restrict__ sl, T *__restrict__ out, int *__restrict__ status) {
+    extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int i = tid; i < g.smem_u64; i += nthr) sm[i] = 0ull;
-    u64 *wtab = sm + g.wtab_off;
+    for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
+    float *wtab = sm + g.wtab_off;
+    unsigned long long *bar = reinterpret_cast<unsigned long long *>(sm + g.bar_off);
+    char *raw = reinterpret_cast<char *>(sm + g.raw_off);
+    unsigned parity = 0;
     const int L = g.L, nlv = g.lvl_start[L + 1];
+    const int nlevel_items = g.NPL * nlv, nitems = nlevel_items + g.NPL * g.nbase;
     const size_t HW = (size_t)g.H * g.W;
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    // this thread's base tile never changes: decode it once
-    const int bi = nthr - 1 - tid;
-    const bool has_base = bi < g.NPP * g.nbase;
-    int bslot = 0, tyy = 0, txx = 0;
-    if (has_base) {
-        bslot = fdiv(bi, g.d_nbase);
-        const int r = bi - bslot * g.nbase;
-        tyy = fdiv(r, g.d_tx[0]);
-        txx = r - tyy * g.tx[0];
-    }
-    const u64 *base_src = sm + (size_t)bslot * g.slot_stride + g.offA[0] + 4 * tyy * g.pitch[0] + 2 * txx;
-    int cp_prev = -1;
+    int c_prev = -1;
     __syncthreads();
+    if (g.bulk && tid == 0) {
+        mbar_init(bar, 1);
+        fence_async_smem();
+        const int c0 = u_begin / g.bgroups;
+        issue_unit_copies<T>(bar, raw, g, x, nullptr, c0, u_begin - c0 * g.bgroups);
+    }
+    __syncthreads();
+    WT_TICK_INIT
     for (int u = u_begin; u < u_end; ++u) {
-        const int cp = u / g.bgroups, bg = u - cp * g.bgroups;
-        const int cA = 2 * cp;
-        const bool hasB = cA + 1 < g.C;
-        if (cp != cp_prev) {  // units are channel-pair major: the table survives all images of a pair
-            build_weight_table(wtab, g, cA, hasB, FLIP, w0, s0, FLIP ? nullptr : b0, wl, sl);
-            cp_prev = cp;
+        const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
+        WT_TICK(0);
+        if (c != c_prev) {  // units are channel-major: the table survives all images of a channel
+            build_weight_table(wtab, g, c, FLIP, w0, s0, FLIP ? nullptr : b0, wl, sl);
+            c_prev = c;
         }
-        stage_input<T>(sm, g, g.offA, x, cA, hasB, bg);
+        WT_TICK(1);
+        int lnext;
+        if (g.bulk) {
+            const bool ok = mbar_wait(bar, parity);
+            parity ^= 1u;
+            if (__syncthreads_or(!ok)) {  // a copy never landed: flag it, let it have one more bounded wait, stop
+                if (tid == 0) atomicExch(status, 1);
+                if (!ok) mbar_wait(bar, parity ^ 1u);
+                return;
+            }
+            WT_TICK(8);
+            lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, bg);
+        } else {
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg);
+        }
+        WT_TICK(2);
         __syncthreads();
-        for (int l = 2; l <= L; ++l) {
+        if (g.bulk && tid == 0 && u + 1 < u_end) {  // the raw buffer is free again: fetch the next unit behind the math
+            fence_async_smem();
+            const int cn = (u + 1) / g.bgroups;
+            issue_unit_copies<T>(bar, raw, g, x, nullptr, cn, (u + 1) - cn * g.bgroups);
+        }
+        WT_TICK(3);
+        for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
             __syncthreads();
         }
-        // ---- level tiles: Z^l = Wfold^l (*) Y^l
-        for (int it = tid; it < g.NPP * nlv; it += nthr) {
-            const int slot = fdiv(it, g.d_nlv);
-            int l, sub, ty2, tx2;
-            decode_level_item(g, it - slot * nlv, l, sub, ty2, tx2);
-            u64 *S = sm + (size_t)slot * g.slot_stride;
-            const int pl = g.pitch[l];
-            u64 w[KK];
-            load_weights(wtab + (1 + (l - 1) * 4 + sub) * WT_STRIDE, w);
-            u64 acc[4][4];
-            conv_tile(S + g.offA[l] + sub * g.rows[l] * pl + 4 * ty2 * pl + 2 * tx2, pl, w, acc);
-            const int zp = g.zpitch[l];
-            u64 *z = S + g.offZ[l] + sub * g.zrows[l] * zp + 4 * ty2 * zp + 4 * tx2;
-            const int zr_left = g.zrows[l] - 4 * ty2;
-            const bool c0 = 4 * tx2 < zp, c1 = 4 * tx2 + 2 < zp;
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                if (r < zr_left) {
-                    ulonglong2 *zr = reinterpret_cast<ulonglong2 *>(z + r * zp);
-                    if (c0) zr[0] = make_ulonglong2(acc[r][0], acc[r][1]);
-                    if (c1) zr[1] = make_ulonglong2(acc[r][2], acc[r][3]);
-                }
-            }
-        }
-        // ---- base tile (at most one per thread), kept in registers across the barrier
-        u64 acc[4][4];
-        u64 bias2 = 0ull;
-        if (has_base) {
-            u64 w[KK];
-            load_weights(wtab, w);
-            conv_tile(base_src, g.pitch[0], w, acc);
-            bias2 = wtab[KK];
-        }
-        __syncthreads();
-        if (has_base) {
-            const u64 *S = sm + (size_t)bslot * g.slot_stride;
-            // Proposition 2, level 1: coefficient (2ty+ci, 2tx+cj) feeds pixels (2ci+by, 2cj+bx) of the tile
-            if (L >= 1) {
-                const u64 half = pk(0.5f, 0.5f);
-                const int zp = g.zpitch[1], zs = g.zrows[1] * zp;
-                const u64 *z = S + g.offZ[1] + (2 * tyy) * zp + 2 * txx;
-#pragma unroll
-                for (int ci = 0; ci < 2; ++ci) {
-                    const ulonglong2 ll = *reinterpret_cast<const ulonglong2 *>(z + ci * zp);
-                    const ulonglong2 lh = *reinterpret_cast<const ulonglong2 *>(z + zs + ci * zp);
-                    const ulonglong2 hl = *reinterpret_cast<const ulonglong2 *>(z + 2 * zs + ci * zp);
-                    const ulonglong2 hh = *reinterpret_cast<const ulonglong2 *>(z + 3 * zs + ci * zp);
-#pragma unroll
-                    for (int cj = 0; cj < 2; ++cj) {
-                        const u64 LLv = cj ? ll.y : ll.x, LHv = cj ? lh.y : lh.x, HLv = cj ? hl.y : hl.x,
-                                  HHv = cj ? hh.y : hh.x;
-                        const u64 pp = add2(LLv, LHv), pm = sub2(LLv, LHv), qp = add2(HLv, HHv), qm = sub2(HLv, HHv);
-                        acc[2 * ci][2 * cj] = fma2(half, add2(pp, qp), acc[2 * ci][2 * cj]);
-                        acc[2 * ci][2 * cj + 1] = fma2(half, sub2(pp, qp), acc[2 * ci][2 * cj + 1]);
-                        acc[2 * ci + 1][2 * cj] = fma2(half, add2(pm, qm), acc[2 * ci + 1][2 * cj]);
-                        acc[2 * ci + 1][2 * cj + 1] = fma2(half, sub2(pm, qm), acc[2 * ci + 1][2 * cj + 1]);
-                    }
-                }
-            }
-            if (L >= 2) {
-                // levels >= 3: the whole tile sits in one quadrant of the coefficient's block
-                u64 deep = bias2;
-                float scale = 0.25f;
-                for (int l = 3; l <= L; ++l) {
-                    scale *= 0.5f;
-                    const int zp = g.zpitch[l], zs = g.zrows[l] * zp;
-                    const u64 *z = S + g.offZ[l] + (tyy >> (l - 2)) * zp + (txx >> (l - 2));
-                    const float sy = ((tyy >> (l - 3)) & 1) ? -1.f : 1.f, sx = ((txx >> (l - 3)) & 1) ? -1.f : 1.f;
-                    const u64 sy2 = pk(sy, sy), sx2 = pk(sx, sx);
-                    const u64 p = fma2(sy2, z[zs], z[0]), q = fma2(sy2, z[3 * zs], z[2 * zs]);
-                    deep = fma2(pk(scale, scale), fma2(sx2, q, p), deep);
-                }
-                // level 2: coefficient (ty, tx); pixel (r, c) of the tile takes signs from (r>>1, c>>1)
-                const int zp = g.zpitch[2], zs = g.zrows[2] * zp;
-                const u64 *z = S + g.offZ[2] + tyy * zp + txx;
-                const u64 LLv = z[0], LHv = z[zs], HLv = z[2 * zs], HHv = z[3 * zs];
-                const u64 pp = add2(LLv, LHv), pm = sub2(LLv, LHv), qp = add2(HLv, HHv), qm = sub2(HLv, HHv);
-                const u64 quarter = pk(0.25f, 0.25f);
-                u64 t2[2][2];
-                t2[0][0] = fma2(quarter, add2(pp, qp), deep);
-                t2[0][1] = fma2(quarter, sub2(pp, qp), deep);
-                t2[1][0] = fma2(quarter, add2(pm, qm), deep);
-                t2[1][1] = fma2(quarter, sub2(pm, qm), deep);
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) acc[r][c] = add2(acc[r][c], t2[r >> 1][c >> 1]);
+        WT_TICK(4);
+        // ---- one item list: level tiles (Z^l = Wfold^l (*) Y^l) first, base tiles last; a thread's last
+        //      item may be a base tile, which stays in registers across the barrier
+        float acc[TH][4];
+        int bslot = 0, tyy = 0, txx = 0;
+        bool has_base = false;
+        for (int it = tid; it < nitems; it += nthr) {
+            const float *src;
+            const float *wt;
+            int pitch, l = 0, sub = 0;
+            const bool is_level = it < nlevel_items;
+            if (is_level) {
+                bslot = fdiv(it, g.d_nlv);
+                decode_level_item(g, it - bslot * nlv, l, sub, tyy, txx);
+                pitch = g.pitch[l];
+                src = sm + (size_t)bslot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * tyy * pitch + 4 * txx;
+                wt = wtab + (1 + (l - 1) * 4 + sub) * WT_STRIDE;
             } else {
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) acc[r][c] = add2(acc[r][c], bias2);
+                const int bi = it - nlevel_items;
+                bslot = fdiv(bi, g.d_nbase);
+                const int r = bi - bslot * g.nbase;
+                tyy = fdiv(r, g.d_tx[0]);
+                txx = r - tyy * g.tx[0];
+                pitch = g.pitch[0];
+                src = sm + (size_t)bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
+                wt = wtab;
+                has_base = true;
             }
-            const int b = bg * g.NPP + bslot;
+            float w[KK];
+            load_weights(wt, w);
+            conv_tile(src, pitch, w, acc);
+            if (is_level) {
+                const int zp = g.zpitch[l];
+                if (4 * txx < zp) {
+                    float *z = sm + (size_t)bslot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * tyy * zp + 4 * txx;
+                    const int zr_left = g.zrows[l] - TH * tyy;
+#pragma unroll
+                    for (int r = 0; r < TH; ++r)
+                        if (r < zr_left) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+                }
+            }
+        }
+        const float bias = wtab[KK];
+        WT_TICK(5);
+        __syncthreads();
+        WT_TICK(6);
+        if (has_base) {
+            const float *S = sm + (size_t)bslot * g.slot_stride;
+#pragma unroll
+            for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, bias, &acc[4 * hb]);
+            const int b = bg * g.NPL + bslot;
             if (b < g.B) {
-                T *oa = out + ((size_t)b * g.C + cA) * HW + (size_t)(4 * tyy) * g.W + 4 * txx;
+                T *oa = out + ((size_t)b * g.C + c) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
                 const bool vec = g.vec && (4 * txx + 3 < g.W);
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if (4 * tyy + r < g.H) {
-                        float a0, a1, a2, a3, b0_, b1, b2, b3;
-                        upk(acc[r][0], a0, b0_);
-                        upk(acc[r][1], a1, b1);
-                        upk(acc[r][2], a2, b2);
-                        upk(acc[r][3], a3, b3);
-                        store_row4<T>(oa + (size_t)r * g.W, 4 * txx, g.W, vec, a0, a1, a2, a3);
-                        if (hasB) store_row4<T>(oa + HW + (size_t)r * g.W, 4 * txx, g.W, vec, b0_, b1, b2, b3);
-                    }
-                }
+                for (int r = 0; r < TH; ++r)
+                    if (TH * tyy + r < g.H) store_row4(oa + (size_t)r * g.W, 4 * txx, g.W, vec, acc[r]);
             }
         }
+        WT_TICK(7);
         // The next unit's staging overwrites x / Y (last read before the barrier above) and possibly the
-        // weight table (bias already copied to a register); Z is next written after the staging barriers.
+        // weight table (bias already in a register); Z is next written after the staging barriers.
     }
 }
 
 // ------------------------------------------------------------------ weight-gradient kernel
 // dWfold^l[u,v] += sum_{i,j} D^l[i,j] Y^l[i+u-2, j+v-2] (and the base class with grad_out and x), Sec. 2.2.
 // Thread t serves class cls(t) only (class-major allocation thr_start[]); accumulators persist over all
-// units of a channel pair and are flushed to `part0` / `partl` when the pair changes.
-template <typename T>
-__global__ void __launch_bounds__(MAX_THREADS, 1)
+// units of a channel and are flushed to `part0` / `partl` when the channel changes.
+template <typename T, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
 plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
-                   float *__restrict__ part0, float *__restrict__ partl /* level l at l*C*np*100 */) {
-    extern __shared__ __align__(16) u64 sm[];
+                   float *__restrict__ part0, float *__restrict__ partl /* level l at l*C*np*100 */,
+                   int *__restrict__ status) {
+    extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int i = tid; i < g.smem_u64; i += nthr) sm[i] = 0ull;
+    for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
+    unsigned long long *bar = reinterpret_cast<unsigned long long *>(sm + g.bar_off);
+    char *raw = reinterpret_cast<char *>(sm + g.raw_off);
+    const int arrays_floats = g.raw_off;  // haloed arrays (and reduction scratch) end where the raw buffer starts
+    unsigned parity = 0;
     const int L = g.L, ncls = 1 + 4 * L;
     int cls = 0;
     while (cls < ncls && tid >= g.thr_start[cls + 1]) ++cls;
@@ -592,121 +663,137 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     const int lvl = active ? (cls == 0 ? 0 : 1 + ((cls - 1) >> 2)) : 0, sub = (cls - 1) & 3;
     const int kth = active ? tid - g.thr_start[cls] : 0, nth = active ? g.thr_start[cls + 1] - g.thr_start[cls] : 1;
     const int ntile = g.tx[lvl] * g.ty[lvl];
-    const int pl = g.pitch[lvl], hl = pl >> 1;
+    const int pl = g.pitch[lvl];
     const int suboff = (lvl == 0 ? 0 : sub * g.rows[lvl] * pl);
-    u64 acc[KK], gsum = 0ull;
+    float acc[KK], gsum = 0.f;
 #pragma unroll
-    for (int t = 0; t < KK; ++t) acc[t] = 0ull;
+    for (int t = 0; t < KK; ++t) acc[t] = 0.f;
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
     __syncthreads();
+    if (g.bulk && tid == 0) {
+        mbar_init(bar, 1);
+        fence_async_smem();
+        const int c0 = u_begin / g.bgroups;
+        issue_unit_copies<T>(bar, raw, g, x, go, c0, u_begin - c0 * g.bgroups);
+    }
+    __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
-        const int cp = u / g.bgroups, bg = u - cp * g.bgroups;
-        const int cA = 2 * cp;
-        const bool hasB = cA + 1 < g.C;
-        stage_input<T>(sm, g, g.offA, x, cA, hasB, bg);
-        stage_input<T>(sm, g, g.offG, go, cA, hasB, bg);
+        const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
+        int lnext;
+        if (g.bulk) {
+            const bool ok = mbar_wait(bar, parity);
+            parity ^= 1u;
+            if (__syncthreads_or(!ok)) {
+                if (tid == 0) atomicExch(status, 1);
+                if (!ok) mbar_wait(bar, parity ^ 1u);
+                return;
+            }
+            const T *rx = reinterpret_cast<const T *>(raw);
+            const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.raw_slot_bytes);
+            lnext = stage_input<T, true>(sm, g, g.offA, rx, c, bg);
+            stage_input<T, true>(sm, g, g.offG, rg, c, bg);
+        } else {
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg);
+            stage_input<T, false>(sm, g, g.offG, go, c, bg);
+        }
         __syncthreads();
-        for (int l = 2; l <= L; ++l) {
+        if (g.bulk && tid == 0 && u + 1 < u_end) {
+            fence_async_smem();
+            const int cn = (u + 1) / g.bgroups;
+            issue_unit_copies<T>(bar, raw, g, x, go, cn, (u + 1) - cn * g.bgroups);
+        }
+        for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
             stage_level(sm, g, g.offG, l);
             __syncthreads();
         }
         if (active) {
-            for (int it = kth; it < g.NPP * ntile; it += nth) {
+            for (int it = kth; it < g.NPL * ntile; it += nth) {
                 const int slot = fdiv(it, g.d_nt[lvl]), r = it - slot * ntile;
                 const int tyy = fdiv(r, g.d_tx[lvl]), txx = r - tyy * g.tx[lvl];
-                const u64 *S = sm + (size_t)slot * g.slot_stride;
-                const u64 *ysrc = S + g.offA[lvl] + suboff + 4 * tyy * pl + 2 * txx;
-                // D tile = columns 4tx+2..4tx+5 of rows 4ty+2..: chunk 2tx+1 (odd half) and chunk 2tx+2 (even half)
-                const u64 *dsrc = S + g.offG[lvl] + suboff + (4 * tyy + 2) * pl + 2 * txx;
-                u64 d[4][4];
+                const float *S = sm + (size_t)slot * g.slot_stride;
+                const float *ysrc = S + g.offA[lvl] + suboff + TH * tyy * pl + 4 * txx;
+                // D tile = columns 4tx+2..4tx+5 of rows TH*ty+2.. (8-byte aligned)
+                const float *dsrc = S + g.offG[lvl] + suboff + (TH * tyy + 2) * pl + 4 * txx + 2;
+                float d[TH][4];
 #pragma unroll
-                for (int rr = 0; rr < 4; ++rr) {
-                    const ulonglong2 q0 = *reinterpret_cast<const ulonglong2 *>(dsrc + rr * pl + hl);
-                    const ulonglong2 q1 = *reinterpret_cast<const ulonglong2 *>(dsrc + rr * pl + 2);
+                for (int rr = 0; rr < TH; ++rr) {
+                    const float2 q0 = *reinterpret_cast<const float2 *>(dsrc + rr * pl);
+                    const float2 q1 = *reinterpret_cast<const float2 *>(dsrc + rr * pl + 2);
                     d[rr][0] = q0.x; d[rr][1] = q0.y; d[rr][2] = q1.x; d[rr][3] = q1.y;
                 }
                 if (cls == 0) {
 #pragma unroll
-                    for (int rr = 0; rr < 4; ++rr)
+                    for (int rr = 0; rr < TH; ++rr)
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) gsum = add2(gsum, d[rr][c]);
+                        for (int cc = 0; cc < 4; ++cc) gsum += d[rr][cc];
                 }
 #pragma unroll
-                for (int rr = 0; rr < 8; ++rr) {
-                    const u64 *rp = ysrc + rr * pl;
-                    const ulonglong2 q0 = *reinterpret_cast<const ulonglong2 *>(rp);
-                    const ulonglong2 q1 = *reinterpret_cast<const ulonglong2 *>(rp + hl);
-                    const ulonglong2 q2 = *reinterpret_cast<const ulonglong2 *>(rp + 2);
-                    const ulonglong2 q3 = *reinterpret_cast<const ulonglong2 *>(rp + hl + 2);
-                    const u64 in[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
+                for (int rr = 0; rr < TH + 4; ++rr) {
+                    const float4 q0 = *reinterpret_cast<const float4 *>(ysrc + rr * pl);
+                    const float4 q1 = *reinterpret_cast<const float4 *>(ysrc + rr * pl + 4);
+                    const float in[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
                     for (int uu = 0; uu < 5; ++uu) {
                         const int dr = rr - uu;
-                        if (dr >= 0 && dr < 4) {
+                        if (dr >= 0 && dr < TH) {
 #pragma unroll
                             for (int v = 0; v < 5; ++v)
 #pragma unroll
-                                for (int c = 0; c < 4; ++c) acc[uu * 5 + v] = fma2(d[dr][c], in[c + v], acc[uu * 5 + v]);
+                                for (int cc = 0; cc < 4; ++cc) acc[uu * 5 + v] = fmaf(d[dr][cc], in[cc + v], acc[uu * 5 + v]);
                         }
                     }
                 }
             }
         }
         __syncthreads();
-        const bool last_of_pair = (u + 1 == u_end) || ((u + 1) / g.bgroups != cp);
-        if (last_of_pair) {
-            // block tree through shared memory: every thread parks its 26 packed sums, then one thread
-            // per (class, tap) adds its class's threads in index order
-            u64 *scr = sm;
+        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_bg) != c);
+        if (last_of_channel) {
+            // block tree through shared memory: every thread parks its 26 sums in the (now idle) array
+            // region, then one thread per (class, tap) adds its class's threads in index order
+            float *scr = sm;
 #pragma unroll
             for (int t = 0; t < KK; ++t) scr[(size_t)tid * (KK + 1) + t] = acc[t];
             scr[(size_t)tid * (KK + 1) + KK] = gsum;
             __syncthreads();
-            const int slotp = blockIdx.x - block_of_unit((long long)cp * g.bgroups, gridDim.x, g.units);
+            const int slotp = blockIdx.x - block_of_unit((long long)c * g.bgroups, gridDim.x, g.units);
             for (int e = tid; e < ncls * (KK + 1); e += nthr) {
                 const int c2 = e / (KK + 1), t = e - c2 * (KK + 1);
                 if (c2 > 0 && t == KK) continue;
-                u64 s = 0ull;
-                for (int th = g.thr_start[c2]; th < g.thr_start[c2 + 1]; ++th) s = add2(s, scr[(size_t)th * (KK + 1) + t]);
-                float sa, sb;
-                upk(s, sa, sb);
+                float s = 0.f;
+                for (int th = g.thr_start[c2]; th < g.thr_start[c2 + 1]; ++th) s += scr[(size_t)th * (KK + 1) + t];
                 if (c2 == 0) {
-                    part0[((size_t)cA * g.np + slotp) * (KK + 1) + t] = sa;
-                    if (hasB) part0[((size_t)(cA + 1) * g.np + slotp) * (KK + 1) + t] = sb;
+                    part0[((size_t)c * g.np + slotp) * (KK + 1) + t] = s;
                 } else {
                     const int l = (c2 - 1) >> 2, sb_ = (c2 - 1) & 3;
-                    float *pl_ = partl + (size_t)l * g.C * g.np * 4 * KK;
-                    pl_[(((size_t)cA * g.np + slotp) * 4 + sb_) * KK + t] = sa;
-                    if (hasB) pl_[(((size_t)(cA + 1) * g.np + slotp) * 4 + sb_) * KK + t] = sb;
+                    partl[(size_t)l * g.C * g.np * 4 * KK + (((size_t)c * g.np + slotp) * 4 + sb_) * KK + t] = s;
                 }
             }
             __syncthreads();
-            for (int i = tid; i < g.smem_u64; i += nthr) sm[i] = 0ull;  // restore the zero halos
+            for (int i = tid; i < arrays_floats; i += nthr) sm[i] = 0.f;  // restore the zero halos (raw buffer untouched)
 #pragma unroll
-            for (int t = 0; t < KK; ++t) acc[t] = 0ull;
-            gsum = 0ull;
+            for (int t = 0; t < KK; ++t) acc[t] = 0.f;
+            gsum = 0.f;
             __syncthreads();
         }
     }
 }
 
 // ------------------------------------------------------------------ host-side planning
-inline void fill_common(Geom &g, int B, int C, int H, int W, int L) {
+inline void fill_common(Geom &g, int B, int C, int H, int W, int L, int elem_bytes) {
     g.B = B; g.C = C; g.H = H; g.W = W; g.L = L;
     g.Hl[0] = H; g.Wl[0] = W;
     for (int l = 1; l <= MAXL; ++l) { g.Hl[l] = (g.Hl[l - 1] + 1) / 2; g.Wl[l] = (g.Wl[l - 1] + 1) / 2; }
     for (int l = 0; l <= L; ++l) {
-        g.rows[l] = pad4(g.Hl[l]) + 4;
-        g.pitch[l] = pad4(g.Wl[l]) + 4;
-        g.ty[l] = pad4(g.Hl[l]) / 4;
+        g.ty[l] = (g.Hl[l] + TH - 1) / TH;
         g.tx[l] = pad4(g.Wl[l]) / 4;
+        g.rows[l] = g.ty[l] * TH + 4;
+        g.pitch[l] = pad4(g.Wl[l]) + 4;
     }
     g.nbase = g.tx[0] * g.ty[0];
     g.lvl_start[0] = 0; g.lvl_start[1] = 0;
     for (int l = 1; l <= L; ++l) g.lvl_start[l + 1] = g.lvl_start[l] + 4 * g.tx[l] * g.ty[l];
-    g.ncp = (C + 1) / 2;
     g.vec = (L >= 1 && (W & 3) == 0) ? 1 : 0;
     if (L >= 1) {
         const int prow = g.vec ? W / 4 : g.Wl[1];
@@ -726,22 +813,41 @@ inline void fill_common(Geom &g, int B, int C, int H, int W, int L) {
     }
     g.d_nlv = make_fastdiv(g.lvl_start[L + 1]);
     g.d_nbase = make_fastdiv(g.nbase);
+    g.npatch4 = ((H + 3) / 4) * (W / 4 > 0 ? W / 4 : 1);
+    g.d_npatch4 = make_fastdiv(g.npatch4);
+    // bulk prefetch needs 16-byte aligned plane starts and sizes
+    g.plane_bytes = H * W * elem_bytes;
+    g.bulk = (g.plane_bytes % 16 == 0) ? 1 : 0;
+    g.raw_slot_bytes = g.plane_bytes;
 }
 
-// Slot layout; returns float2 count per slot.  with_g: second copy of the input pyramid (grad_out);
-// with_z: the conv-output arrays.
+// Tail of the shared-memory layout: [arrays][weight table][raw planes (bulk only)][mbarrier].  Returns floats.
+inline long long finish_layout(Geom &g, long long arrays_floats, int wtab_floats, int raw_tensors, bool use_bulk) {
+    long long off = pad4((int)arrays_floats);
+    g.wtab_off = (int)off;
+    off += pad4(wtab_floats);
+    g.raw_off = (int)off;
+    if (use_bulk) off += (long long)raw_tensors * g.NPL * g.raw_slot_bytes / 4;
+    off = pad4((int)off);
+    g.bar_off = (int)off;
+    return off + 4;
+}
+
+// Slot layout; returns floats per slot.  with_g: second copy of the input pyramid (grad_out); with_z:
+// the conv-output arrays.
 inline int layout_slot(Geom &g, bool with_g, bool with_z) {
     int off = 0;
     for (int l = 0; l <= g.L; ++l) { g.offA[l] = off; off += (l == 0 ? 1 : 4) * g.rows[l] * g.pitch[l]; }
     for (int l = 0; l <= g.L; ++l) { g.offG[l] = off; if (with_g) off += (l == 0 ? 1 : 4) * g.rows[l] * g.pitch[l]; }
+    const int padH = g.ty[0] * TH, padW = g.tx[0] * 4;  // pixels the base tiles cover
     for (int l = 1; l <= g.L; ++l) {
-        // only the coefficients the (padded) 4x4 pixel tiles read in the synthesis are kept
-        const int zr = ((pad4(g.H) - 1) >> l) + 1;
-        const int zc = ((((pad4(g.W) - 1) >> l) + 1) + 1) & ~1;
+        // only the coefficients the (padded) base tiles read in the synthesis are kept
+        const int zr = ((padH - 1) >> l) + 1;
+        const int zc = pad4(((padW - 1) >> l) + 1);
         g.zrows[l] = zr; g.zpitch[l] = zc; g.offZ[l] = off;
         if (with_z) off += 4 * zr * zc;
     }
-    return (off + 1) & ~1;
+    return pad4(off);
 }
 
 inline double partition_eff(int units, int nblocks) {
@@ -749,70 +855,78 @@ inline double partition_eff(int units, int nblocks) {
     return (double)units / ((double)per * nblocks);
 }
 
-// Forward plan: maximise (tile-slot use) x (threads resident) x (phase overlap) x (tail) over NPP, T, blocks/SM.
-// `tune` (0 = automatic): bits 0-5 threads/32, bits 6-7 blocks per SM, bits 8-14 plane pairs per unit.
-inline bool plan_forward(int B, int C, int H, int W, int L, Geom &best, unsigned tune = 0) {
-    const int fT = (tune & 63) * 32, fBps = (tune >> 6) & 3, fNpp = (tune >> 8) & 127;
+// Forward plan.  `tune` (0 = automatic): bits 0-4 threads/32, bits 5-7 blocks per SM, bits 8-13 planes per unit.
+inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    const int fT = (tune & 31) * 32, fBps = (tune >> 5) & 7, fNpl = (tune >> 8) & 63;
+    const bool no_bulk = (tune >> 23) & 1;
     Geom g = {};
-    fill_common(g, B, C, H, W, L);
+    fill_common(g, B, C, H, W, L, elem_bytes);
     const int slot = layout_slot(g, false, true);
     const int M = g.lvl_start[L + 1] + g.nbase;
     const int wtab = (1 + 4 * L) * WT_STRIDE;
     bool found = false;
     best.score = -1.0;
-    for (int npp = 1; npp <= 64; ++npp) {
-        if (npp > 1 && npp > B) break;
-        if (fNpp && npp != fNpp) continue;
-        const long long smem_u64 = (long long)npp * slot + ((wtab + 1) & ~1);
-        const long long bytes = smem_u64 * 8;
-        if (bytes > SMEM_LIMIT) break;
+    for (int npl = 1; npl <= 64; ++npl) {
+        if (npl > 1 && npl > B) break;
+        if (fNpl && npl != fNpl) continue;
+        for (int use_bulk = (g.bulk && !no_bulk) ? 1 : 0; use_bulk >= 0; --use_bulk) {
+        Geom cg = g;
+        cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
+        const long long smem_floats = finish_layout(cg, (long long)npl * slot, wtab, 1, use_bulk);
+        const long long bytes = smem_floats * 4;
+        if (bytes > SMEM_LIMIT) continue;
         for (int T = 64; T <= MAX_THREADS; T += 32) {
-            if (npp * g.nbase > T) continue;
+            if (npl * g.nbase > T) continue;  // at most one base tile per thread
             if (fT && T != fT) continue;
-            for (int bps = 1; bps <= 4; ++bps) {
-                if (bps * T > 512) continue;
+            for (int bps = 1; bps <= 6; ++bps) {
+                if (bps * T > 768) continue;  // register file: kernels are built for 128 / 84 registers
                 if (fBps && bps != fBps) continue;
                 if (bps * (bytes + 1024) > SMEM_PER_SM) continue;
-                const int rounds = (npp * M + T - 1) / T;
-                const double eff = (double)npp * M / ((double)T * rounds);
-                const int bgroups = (B + npp - 1) / npp, units = g.ncp * bgroups;
+                const int rounds = (npl * M + T - 1) / T;
+                const double eff = (double)npl * M / ((double)T * rounds);
+                const int bgroups = (B + npl - 1) / npl, units = C * bgroups;
                 int nblocks = NUM_SMS * bps;
                 if (nblocks > units) nblocks = units;
-                const double sc = eff * ((double)bps * T / 512.0) * (bps >= 2 ? 1.0 : 0.9) *
-                                  partition_eff(units, nblocks) * ((double)B / ((double)bgroups * npp)) *
-                                  (rounds <= 3 ? 1.0 : 0.97);
+                // thread-slot use x resident warps (about 16 hide the latency-bound phases) x phase overlap
+                double occ = (double)bps * T / 512.0;
+                if (occ > 1.0) occ = 1.0;
+                const double overlap = bps >= 4 ? 1.0 : (bps == 3 ? 0.95 : (bps == 2 ? 0.8 : 0.55));
+                const double sc = eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) *
+                                  partition_eff(units, nblocks) * ((double)B / ((double)bgroups * npl));
                 if (sc > best.score + 1e-9) {
-                    best = g;
-                    best.NPP = npp; best.slot_stride = slot; best.wtab_off = npp * slot;
-                    best.smem_u64 = (int)smem_u64; best.bgroups = bgroups; best.units = units;
+                    best = cg;
+                    best.smem_floats = (int)smem_floats; best.bgroups = bgroups; best.units = units;
+                    best.d_bg = make_fastdiv(bgroups);
                     best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                     found = true;
                 }
             }
         }
+        }
     }
     return found;
 }
 
-// Weight-gradient plan: one block per SM; per class c with n_c tiles (x NPP) allocate ceil(n_c NPP / rounds)
-// threads, smallest `rounds` that fits 512 threads.
-inline bool plan_wgrad(int B, int C, int H, int W, int L, Geom &best, unsigned tune = 0) {
-    const int fNpp = (tune >> 15) & 127;
+// Weight-gradient plan: per class c with n_c tiles (x NPL) allocate ceil(n_c NPL / rounds) threads, smallest
+// `rounds` that fits the thread limit.  tune bits 14-19: planes per unit, bits 20-22: blocks per SM.
+inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    const int fNpl = (tune >> 14) & 63, fBps = (tune >> 20) & 7;
+    const bool no_bulk = (tune >> 23) & 1;
     Geom g = {};
-    fill_common(g, B, C, H, W, L);
+    fill_common(g, B, C, H, W, L, elem_bytes);
     const int slot = layout_slot(g, true, false);
     const int ncls = 1 + 4 * L;
     bool found = false;
     best.score = -1.0;
-    for (int npp = 1; npp <= 64; ++npp) {
-        if (npp > 1 && npp > B) break;
-        if (fNpp && npp != fNpp) continue;
+    for (int npl = 1; npl <= 64; ++npl) {
+        if (npl > 1 && npl > B) break;
+        if (fNpl && npl != fNpl) continue;
         for (int rounds = 1; rounds <= 64; ++rounds) {
             int thr[4 * MAXL + 2];
             int tot = 0, work = 0;
             for (int c = 0; c < ncls; ++c) {
                 const int l = c == 0 ? 0 : 1 + ((c - 1) >> 2);
-                const int n = g.tx[l] * g.ty[l] * npp;
+                const int n = g.tx[l] * g.ty[l] * npl;
                 thr[c] = tot;
                 tot += (n + rounds - 1) / rounds;
                 work += n;
@@ -820,85 +934,130 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, Geom &best, unsigned t
             thr[ncls] = tot;
             if (tot > MAX_THREADS) continue;
             const int T = (tot + 31) & ~31;
-            long long smem_u64 = (long long)npp * slot;
+            long long arrays = (long long)npl * slot;
             const long long scratch = (long long)T * (KK + 1);
-            if (scratch > smem_u64) smem_u64 = scratch;
-            smem_u64 = (smem_u64 + 1) & ~1LL;
-            if (smem_u64 * 8 > SMEM_LIMIT) break;
-            const int bgroups = (B + npp - 1) / npp, units = g.ncp * bgroups;
-            int nblocks = NUM_SMS;
-            if (nblocks > units) nblocks = units;
-            const double sc = ((double)work / ((double)T * rounds)) * ((double)T / 512.0) *
-                              partition_eff(units, nblocks) * ((double)B / ((double)bgroups * npp));
-            if (sc > best.score + 1e-9) {
-                best = g;
-                best.NPP = npp; best.slot_stride = slot; best.wtab_off = 0; best.smem_u64 = (int)smem_u64;
-                best.bgroups = bgroups; best.units = units; best.nthreads = T; best.nblocks = nblocks;
-                best.blocks_per_sm = 1; best.score = sc;
-                for (int c = 0; c <= ncls; ++c) best.thr_start[c] = thr[c];
-                int np = 1;
-                for (int cp = 0; cp < g.ncp; ++cp) {
-                    const int first = block_of_unit((long long)cp * bgroups, nblocks, units);
-                    const int last = block_of_unit((long long)(cp + 1) * bgroups - 1, nblocks, units);
-                    if (last - first + 1 > np) np = last - first + 1;
+            if (scratch > arrays) arrays = scratch;
+            bool any = false;
+            for (int use_bulk = (g.bulk && !no_bulk) ? 1 : 0; use_bulk >= 0; --use_bulk) {
+                Geom cg = g;
+                cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
+                const long long smem_floats = finish_layout(cg, arrays, 0, 2, use_bulk);
+                const long long bytes = smem_floats * 4;
+                if (bytes > SMEM_LIMIT) continue;
+                any = true;
+                for (int bps = 1; bps <= 4; ++bps) {
+                    if (bps * T > 512) continue;  // 128 registers per thread
+                    if (fBps && bps != fBps) continue;
+                    if (bps * (bytes + 1024) > SMEM_PER_SM) continue;
+                    const int bgroups = (B + npl - 1) / npl, units = C * bgroups;
+                    int nblocks = NUM_SMS * bps;
+                    if (nblocks > units) nblocks = units;
+                    double occ = (double)bps * T / 512.0;
+                    if (occ > 1.0) occ = 1.0;
+                    const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
+                    const double sc = ((double)work / ((double)T * rounds)) * (0.5 + 0.5 * occ) * overlap *
+                                      (use_bulk ? 1.0 : 0.8) * partition_eff(units, nblocks) *
+                                      ((double)B / ((double)bgroups * npl));
+                    if (sc > best.score + 1e-9) {
+                        best = cg;
+                        best.smem_floats = (int)smem_floats;
+                        best.bgroups = bgroups; best.units = units; best.d_bg = make_fastdiv(bgroups);
+                        best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
+                        for (int k = 0; k <= ncls; ++k) best.thr_start[k] = thr[k];
+                        int np = 1;
+                        for (int ch = 0; ch < C; ++ch) {
+                            const int first = block_of_unit((long long)ch * bgroups, nblocks, units);
+                            const int last = block_of_unit((long long)(ch + 1) * bgroups - 1, nblocks, units);
+                            if (last - first + 1 > np) np = last - first + 1;
+                        }
+                        best.np = np;
+                        found = true;
+                    }
                 }
-                best.np = np;
-                found = true;
             }
-            break;  // more rounds with the same NPP only lowers thread use
+            if (!any) break;
+            break;  // more rounds with the same NPL only lowers thread use
         }
     }
     return found;
 }
 
+inline int dtype_bytes(int dtype) { return dtype == 0 ? 4 : 2; }
+
 inline bool supported(int H, int W, int k, int L, int dtype) {
-    (void)dtype;
     if (k != 5) return false;
     Geom g;
-    return plan_forward(2, 2, H, W, L, g) && plan_wgrad(2, 2, H, W, L, g);
+    return plan_forward(2, 2, H, W, L, dtype_bytes(dtype), g) && plan_wgrad(2, 2, H, W, L, dtype_bytes(dtype), g);
 }
 
-inline size_t forward_workspace_bytes(int, int, int, int, int) { return 0; }
-
-// Backward workspace: base partials [C][np][26] then level partials [L][C][np][4][25] (float).
-inline size_t backward_workspace_bytes(int B, int C, int H, int W, int L, unsigned tune = 0) {
+// Workspace: a status word (256 bytes reserved; nonzero after a run = a bounded wait on a copy barrier ran
+// out), then for backward the base partials [C][np][26] and the level partials [L][C][np][4][25] (float).
+constexpr size_t STATUS_BYTES = 256;
+inline size_t forward_workspace_bytes(int, int, int, int, int) { return STATUS_BYTES; }
+inline size_t backward_workspace_bytes(int B, int C, int H, int W, int L, int elem_bytes, unsigned tune = 0) {
     Geom g;
-    if (!plan_wgrad(B, C, H, W, L, g, tune)) return 0;
-    return sizeof(float) * ((size_t)C * g.np * (KK + 1) + (size_t)L * C * g.np * 4 * KK);
+    if (!plan_wgrad(B, C, H, W, L, elem_bytes, g, tune)) return 0;
+    return STATUS_BYTES + sizeof(float) * ((size_t)C * g.np * (KK + 1) + (size_t)L * C * g.np * 4 * KK);
 }
 
-template <typename T>
-cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
-                    const float *wl, const float *sl, T *out, char *, cudaStream_t st, unsigned tune = 0) {
-    Geom g;
-    if (!plan_forward(B, C, H, W, L, g, tune)) return cudaErrorInvalidValue;
-    auto kern = plane_fwd_kernel<T, false>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-    if (e != cudaSuccess) return e;
-    kern<<<g.nblocks, g.nthreads, (size_t)g.smem_u64 * 8, st>>>(g, x, w0, s0, b0, wl, sl, out);
+template <typename T, bool FLIP>
+cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *s0, const float *b0, const float *wl,
+                       const float *sl, T *out, int *status, cudaStream_t st) {
+    cudaError_t e;
+    const size_t smem = (size_t)g.smem_floats * 4;
+#define WT_LAUNCH_FWD(MAXT_, MINB_)                                                                 \
+    {                                                                                               \
+        auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_>;                                        \
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);    \
+        if (e != cudaSuccess) return e;                                                             \
+        kern<<<g.nblocks, g.nthreads, smem, st>>>(g, x, w0, s0, b0, wl, sl, out, status);           \
+    }
+    if (g.nthreads * g.blocks_per_sm <= 512) {
+        if (g.nthreads <= 128) WT_LAUNCH_FWD(128, 4) else WT_LAUNCH_FWD(256, 2)
+    } else {
+        if (g.nthreads <= 128) WT_LAUNCH_FWD(128, 6) else WT_LAUNCH_FWD(256, 3)
+    }
+#undef WT_LAUNCH_FWD
     return cudaGetLastError();
 }
 
 template <typename T>
+cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
+                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tune = 0) {
+    Geom g;
+    if (!plan_forward(B, C, H, W, L, (int)sizeof(T), g, tune)) return cudaErrorInvalidValue;
+    cudaError_t e = cudaMemsetAsync(ws, 0, STATUS_BYTES, st);
+    if (e != cudaSuccess) return e;
+    return launch_fwd<T, false>(g, x, w0, s0, b0, wl, sl, out, reinterpret_cast<int *>(ws), st);
+}
+
+template <typename T>
 cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go, const float *w0, const float *s0,
-                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st, unsigned tune = 0) {
+                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st,
+                     unsigned tune = 0) {
     Geom gw, gf;
-    if (!plan_wgrad(B, C, H, W, L, gw, tune) || !plan_forward(B, C, H, W, L, gf, tune)) return cudaErrorInvalidValue;
-    float *part0 = reinterpret_cast<float *>(ws);
+    if (!plan_wgrad(B, C, H, W, L, (int)sizeof(T), gw, tune) || !plan_forward(B, C, H, W, L, (int)sizeof(T), gf, tune))
+        return cudaErrorInvalidValue;
+    int *status = reinterpret_cast<int *>(ws);
+    float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
     float *partl = part0 + (size_t)C * gw.np * (KK + 1);
-    const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, tune);
-    cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // slots no block writes must read as zero
+    const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
+    cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // status word; partial slots no block writes must read as zero
     if (e != cudaSuccess) return e;
-    auto kw = plane_wgrad_kernel<T>;
-    e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-    if (e != cudaSuccess) return e;
-    kw<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_u64 * 8, st>>>(gw, x, go, part0, partl);
+    const size_t smem = (size_t)gw.smem_floats * 4;
+    if (gw.nthreads <= 128) {
+        auto kw = plane_wgrad_kernel<T, 128, 4>;
+        e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+        if (e != cudaSuccess) return e;
+        kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);
+    } else {
+        auto kw = plane_wgrad_kernel<T, 256, 2>;
+        e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+        if (e != cudaSuccess) return e;
+        kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);
+    }
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    auto kf = plane_fwd_kernel<T, true>;
-    e = cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-    if (e != cudaSuccess) return e;
-    kf<<<gf.nblocks, gf.nthreads, (size_t)gf.smem_u64 * 8, st>>>(gf, go, w0, s0, nullptr, wl, sl, gx);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_fwd<T, true>(gf, go, w0, s0, nullptr, wl, sl, gx, status, st)) != cudaSuccess) return e;
     ep->part0 = part0;
     ep->np0 = gw.np;
     for (int l = 0; l < L; ++l) {

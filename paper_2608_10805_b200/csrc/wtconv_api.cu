@@ -251,7 +251,7 @@ size_t fwd_ws_bytes(const wtconv_desc *d) {
     return make_tiled_plan(d).fwd_bytes;
 }
 size_t bwd_ws_bytes(const wtconv_desc *d) {
-    if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, d->flags >> 8));
+    if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), d->flags >> 8));
     return make_tiled_plan(d).bwd_bytes;
 }
 
@@ -430,5 +430,15 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     d2h(h_gsl, gsl, ps.sl);
     return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
 }
+
+#ifdef WT_PHASE_TIMING
+// working probe only (never part of the shipped library): read and clear the per-phase cycle counters
+int wtconv_debug_phase_cycles(unsigned long long *out16) {
+    cudaDeviceSynchronize();
+    unsigned long long z[32] = {0};
+    if (cudaMemcpyFromSymbol(out16, wt::plane::wt_phase_cycles, sizeof(z)) != cudaSuccess) return 1;
+    return cudaMemcpyToSymbol(wt::plane::wt_phase_cycles, z, sizeof(z)) != cudaSuccess;
+}
+#endif
 
 }  // extern "C"
