@@ -33,7 +33,7 @@ constexpr int NUM_SMS = 148;                 // planning constant (B200); plans 
 constexpr int SMEM_LIMIT = 227 * 1024;       // opt-in dynamic shared memory per block
 constexpr int SMEM_PER_SM = 228 * 1024;      // per SM, 1 KB reserved per resident block
 constexpr int WT_STRIDE = 28;                // floats per class in the weight table (25 taps, 16-byte padded)
-constexpr unsigned WAIT_LIMIT = 1u << 24;    // bounded spin on the copy barrier (never an endless loop)
+constexpr unsigned WAIT_LIMIT = 1u << 20;    // bounded number of (suspending) waits on the copy barrier: never an endless loop
 
 // ------------------------------------------------------------------ bulk-copy (TMA, untiled) helpers
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -51,12 +51,13 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                  "l"(src), "r"(bytes), "r"(smem_addr(bar))
                  : "memory");
 }
-// Bounded wait for phase `parity` of `bar`; false if it did not complete within WAIT_LIMIT polls.
+// Bounded wait for phase `parity` of `bar`: try_wait suspends the thread for a hardware-limited time per call, so
+// waiting costs few instructions; false if the phase did not complete within WAIT_LIMIT calls.
 __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
     const unsigned a = smem_addr(bar);
     for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
         unsigned ok;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok)
                      : "r"(a), "r"(parity)
                      : "memory");
@@ -213,17 +214,18 @@ __device__ __forceinline__ void ld4(const T *p, float (&v)[4]) {
 // halo); images beyond the batch are written as zeros.
 template <typename T, bool RAW>
 __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *off, const T *__restrict__ src, int c,
-                                           int bg) {
-    const int H = g.H, W = g.W;
-    const size_t HW = (size_t)H * W;
+                                           int bg, int srank, int nstagers) {
+    const int H = g.H, W = g.W, HW = H * W;
     const int p0 = g.pitch[0];
-    const size_t slot_elems = RAW ? (size_t)g.raw_slot_bytes / sizeof(T) : 0;
+    const int slot_elems = RAW ? g.raw_slot_bytes / (int)sizeof(T) : 0;
+    const T *gsrc = RAW ? src : src + ((size_t)bg * g.NPL * g.C + c) * HW;  // image bg*NPL of channel c
+    const int img_stride = RAW ? slot_elems : g.C * HW;                      // next image of the unit (elements)
     if (g.L == 0) {
-        for (int e = threadIdx.x; e < g.NPL * H * W; e += blockDim.x) {
-            const int slot = fdiv(e, g.d_npatch), r = e - slot * (H * W), y = fdiv(r, g.d_prow), xx = r - y * W;
-            const int b = bg * g.NPL + slot;
-            const T *pa = RAW ? src + slot * slot_elems + r : src + ((size_t)b * g.C + c) * HW + r;
-            sm[(size_t)slot * g.slot_stride + off[0] + (y + 2) * p0 + xx + 2] = b < g.B ? ld1<T, RAW>(pa) : 0.f;
+        for (int e = srank; e < g.NPL * HW; e += nstagers) {
+            const int slot = fdiv(e, g.d_npatch), r = e - slot * HW, y = fdiv(r, g.d_prow), xx = r - y * W;
+            const bool valid = bg * g.NPL + slot < g.B;
+            sm[slot * g.slot_stride + off[0] + (y + 2) * p0 + xx + 2] =
+                valid ? ld1<T, RAW>(gsrc + (size_t)slot * img_stride + r) : 0.f;
         }
         return 1;
     }
@@ -231,28 +233,28 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
     if (g.vec && g.L >= 2) {
         // work item = 4 rows x 4 columns: four level-1 blocks and the level-2 block above them
         const int p2 = g.pitch[2], sub2 = g.rows[2] * p2;
-        for (int e = threadIdx.x; e < g.NPL * g.npatch4; e += blockDim.x) {
+        for (int e = srank; e < g.NPL * g.npatch4; e += nstagers) {
             const int slot = fdiv(e, g.d_npatch4), r = e - slot * g.npatch4;
             const int i2 = fdiv(r, g.d_prow), q = r - i2 * (int)g.d_prow.d;
-            const int b = bg * g.NPL + slot, y = 4 * i2;
+            const int y = 4 * i2;
             float a[4][4];
 #pragma unroll
             for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) a[rr][cc] = 0.f;
-            if (b < g.B) {
-                const T *pa = (RAW ? src + slot * slot_elems : src + ((size_t)b * g.C + c) * HW) + (size_t)y * W + 4 * q;
+            if (bg * g.NPL + slot < g.B) {
+                const T *pa = gsrc + (size_t)slot * img_stride + y * W + 4 * q;
 #pragma unroll
                 for (int rr = 0; rr < 4; ++rr)
-                    if (y + rr < H) ld4<T, RAW>(pa + (size_t)rr * W, a[rr]);
+                    if (y + rr < H) ld4<T, RAW>(pa + rr * W, a[rr]);
             }
-            float *S = sm + (size_t)slot * g.slot_stride;
-            float *X = S + off[0] + (y + 2) * p0 + 4 * q + 2;  // 8-byte aligned
+            const int S = slot * g.slot_stride;
+            const int xi = S + off[0] + (y + 2) * p0 + 4 * q + 2;  // 8-byte aligned
 #pragma unroll
             for (int rr = 0; rr < 4; ++rr) {
                 if (y + rr < H) {
-                    *reinterpret_cast<float2 *>(X + rr * p0) = make_float2(a[rr][0], a[rr][1]);
-                    *reinterpret_cast<float2 *>(X + rr * p0 + 2) = make_float2(a[rr][2], a[rr][3]);
+                    *reinterpret_cast<float2 *>(&sm[xi + rr * p0]) = make_float2(a[rr][0], a[rr][1]);
+                    *reinterpret_cast<float2 *>(&sm[xi + rr * p0 + 2]) = make_float2(a[rr][2], a[rr][3]);
                 }
             }
             Haar4 h[2][2];
@@ -262,80 +264,80 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
                 for (int bj = 0; bj < 2; ++bj)
                     h[bi][bj] = haar_butterfly(a[2 * bi][2 * bj], a[2 * bi][2 * bj + 1], a[2 * bi + 1][2 * bj],
                                                a[2 * bi + 1][2 * bj + 1]);
-            float *Y = S + off[1] + (2 * i2 + 2) * p1 + 2 * q + 2;
+            const int yi = S + off[1] + (2 * i2 + 2) * p1 + 2 * q + 2;
 #pragma unroll
             for (int bi = 0; bi < 2; ++bi) {
-                *reinterpret_cast<float2 *>(Y + bi * p1) = make_float2(h[bi][0].ll, h[bi][1].ll);
-                *reinterpret_cast<float2 *>(Y + bi * p1 + sub1) = make_float2(h[bi][0].lh, h[bi][1].lh);
-                *reinterpret_cast<float2 *>(Y + bi * p1 + 2 * sub1) = make_float2(h[bi][0].hl, h[bi][1].hl);
-                *reinterpret_cast<float2 *>(Y + bi * p1 + 3 * sub1) = make_float2(h[bi][0].hh, h[bi][1].hh);
+                *reinterpret_cast<float2 *>(&sm[yi + bi * p1]) = make_float2(h[bi][0].ll, h[bi][1].ll);
+                *reinterpret_cast<float2 *>(&sm[yi + bi * p1 + sub1]) = make_float2(h[bi][0].lh, h[bi][1].lh);
+                *reinterpret_cast<float2 *>(&sm[yi + bi * p1 + 2 * sub1]) = make_float2(h[bi][0].hl, h[bi][1].hl);
+                *reinterpret_cast<float2 *>(&sm[yi + bi * p1 + 3 * sub1]) = make_float2(h[bi][0].hh, h[bi][1].hh);
             }
             const Haar4 h2 = haar_butterfly(h[0][0].ll, h[0][1].ll, h[1][0].ll, h[1][1].ll);
-            float *Y2 = S + off[2] + (i2 + 2) * p2 + q + 2;
-            Y2[0] = h2.ll;
-            Y2[sub2] = h2.lh;
-            Y2[2 * sub2] = h2.hl;
-            Y2[3 * sub2] = h2.hh;
+            const int y2 = S + off[2] + (i2 + 2) * p2 + q + 2;
+            sm[y2] = h2.ll;
+            sm[y2 + sub2] = h2.lh;
+            sm[y2 + 2 * sub2] = h2.hl;
+            sm[y2 + 3 * sub2] = h2.hh;
         }
         return 3;
     }
     if (g.vec) {
         // work item = 2 rows x 4 columns: two Haar blocks
-        for (int e = threadIdx.x; e < g.NPL * g.npatch; e += blockDim.x) {
+        for (int e = srank; e < g.NPL * g.npatch; e += nstagers) {
             const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
             const int i = fdiv(r, g.d_prow), q = r - i * (int)g.d_prow.d;
-            const int b = bg * g.NPL + slot, y = 2 * i;
+            const int y = 2 * i;
             const bool y1 = y + 1 < H;
             float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
-            if (b < g.B) {
-                const T *pa = (RAW ? src + slot * slot_elems : src + ((size_t)b * g.C + c) * HW) + (size_t)y * W + 4 * q;
+            if (bg * g.NPL + slot < g.B) {
+                const T *pa = gsrc + (size_t)slot * img_stride + y * W + 4 * q;
                 ld4<T, RAW>(pa, a0);
                 if (y1) ld4<T, RAW>(pa + W, a1);
             }
-            float *S = sm + (size_t)slot * g.slot_stride;
-            float *X = S + off[0] + (y + 2) * p0 + 4 * q + 2;  // 8-byte aligned
-            *reinterpret_cast<float2 *>(X) = make_float2(a0[0], a0[1]);
-            *reinterpret_cast<float2 *>(X + 2) = make_float2(a0[2], a0[3]);
+            const int S = slot * g.slot_stride;
+            const int xi = S + off[0] + (y + 2) * p0 + 4 * q + 2;  // 8-byte aligned
+            *reinterpret_cast<float2 *>(&sm[xi]) = make_float2(a0[0], a0[1]);
+            *reinterpret_cast<float2 *>(&sm[xi + 2]) = make_float2(a0[2], a0[3]);
             if (y1) {
-                *reinterpret_cast<float2 *>(X + p0) = make_float2(a1[0], a1[1]);
-                *reinterpret_cast<float2 *>(X + p0 + 2) = make_float2(a1[2], a1[3]);
+                *reinterpret_cast<float2 *>(&sm[xi + p0]) = make_float2(a1[0], a1[1]);
+                *reinterpret_cast<float2 *>(&sm[xi + p0 + 2]) = make_float2(a1[2], a1[3]);
             }
             const Haar4 ha = haar_butterfly(a0[0], a0[1], a1[0], a1[1]), hb = haar_butterfly(a0[2], a0[3], a1[2], a1[3]);
-            float *Y = S + off[1] + (i + 2) * p1 + 2 * q + 2;
-            *reinterpret_cast<float2 *>(Y) = make_float2(ha.ll, hb.ll);
-            *reinterpret_cast<float2 *>(Y + sub1) = make_float2(ha.lh, hb.lh);
-            *reinterpret_cast<float2 *>(Y + 2 * sub1) = make_float2(ha.hl, hb.hl);
-            *reinterpret_cast<float2 *>(Y + 3 * sub1) = make_float2(ha.hh, hb.hh);
+            const int yi = S + off[1] + (i + 2) * p1 + 2 * q + 2;
+            *reinterpret_cast<float2 *>(&sm[yi]) = make_float2(ha.ll, hb.ll);
+            *reinterpret_cast<float2 *>(&sm[yi + sub1]) = make_float2(ha.lh, hb.lh);
+            *reinterpret_cast<float2 *>(&sm[yi + 2 * sub1]) = make_float2(ha.hl, hb.hl);
+            *reinterpret_cast<float2 *>(&sm[yi + 3 * sub1]) = make_float2(ha.hh, hb.hh);
         }
         return 2;
     }
     // general path: one 2x2 block per work item, scalar loads
     const int W1 = g.Wl[1];
-    for (int e = threadIdx.x; e < g.NPL * g.npatch; e += blockDim.x) {
+    for (int e = srank; e < g.NPL * g.npatch; e += nstagers) {
         const int slot = fdiv(e, g.d_npatch), r = e - slot * g.npatch;
         const int i = fdiv(r, g.d_prow), j = r - i * W1;
-        const int b = bg * g.NPL + slot, y = 2 * i, xx = 2 * j;
+        const int y = 2 * i, xx = 2 * j;
         const bool x1 = xx + 1 < W, y1 = y + 1 < H;
         float a = 0.f, bq = 0.f, cq = 0.f, d = 0.f;
-        if (b < g.B) {
-            const T *pa = (RAW ? src + slot * slot_elems : src + ((size_t)b * g.C + c) * HW) + (size_t)y * W + xx;
+        if (bg * g.NPL + slot < g.B) {
+            const T *pa = gsrc + (size_t)slot * img_stride + y * W + xx;
             a = ld1<T, RAW>(pa);
             if (x1) bq = ld1<T, RAW>(pa + 1);
             if (y1) cq = ld1<T, RAW>(pa + W);
             if (x1 && y1) d = ld1<T, RAW>(pa + W + 1);
         }
-        float *S = sm + (size_t)slot * g.slot_stride;
-        float *X = S + off[0] + (y + 2) * p0 + xx + 2;
-        X[0] = a;
-        if (x1) X[1] = bq;
-        if (y1) X[p0] = cq;
-        if (x1 && y1) X[p0 + 1] = d;
+        const int S = slot * g.slot_stride;
+        const int xi = S + off[0] + (y + 2) * p0 + xx + 2;
+        sm[xi] = a;
+        if (x1) sm[xi + 1] = bq;
+        if (y1) sm[xi + p0] = cq;
+        if (x1 && y1) sm[xi + p0 + 1] = d;
         const Haar4 h = haar_butterfly(a, bq, cq, d);
-        float *Y = S + off[1] + (i + 2) * p1 + j + 2;
-        Y[0] = h.ll;
-        Y[sub1] = h.lh;
-        Y[2 * sub1] = h.hl;
-        Y[3 * sub1] = h.hh;
+        const int yi = S + off[1] + (i + 2) * p1 + j + 2;
+        sm[yi] = h.ll;
+        sm[yi + sub1] = h.lh;
+        sm[yi + 2 * sub1] = h.hl;
+        sm[yi + 3 * sub1] = h.hh;
     }
     return 2;
 }
@@ -365,16 +367,16 @@ __device__ __forceinline__ void stage_level(float *sm, const Geom &g, const int 
     const int pp = g.pitch[l - 1], pl = g.pitch[l], subl = g.rows[l] * pl;
     for (int e = threadIdx.x; e < g.NPL * n; e += blockDim.x) {
         const int slot = fdiv(e, g.d_lvl[l]), r = e - slot * n, i = fdiv(r, g.d_lvlw[l]), j = r - i * Wl;
-        float *S = sm + (size_t)slot * g.slot_stride;
-        const float *src = S + off[l - 1] + (2 * i + 2) * pp + 2 * j + 2;  // even column: 8-byte aligned
-        const float2 top = *reinterpret_cast<const float2 *>(src);
-        const float2 bot = *reinterpret_cast<const float2 *>(src + pp);
+        const int S = slot * g.slot_stride;
+        const int si = S + off[l - 1] + (2 * i + 2) * pp + 2 * j + 2;  // even column: 8-byte aligned
+        const float2 top = *reinterpret_cast<const float2 *>(&sm[si]);
+        const float2 bot = *reinterpret_cast<const float2 *>(&sm[si + pp]);
         const Haar4 h = haar_butterfly(top.x, top.y, bot.x, bot.y);
-        float *Y = S + off[l] + (i + 2) * pl + j + 2;
-        Y[0] = h.ll;
-        Y[subl] = h.lh;
-        Y[2 * subl] = h.hl;
-        Y[3 * subl] = h.hh;
+        const int yi = S + off[l] + (i + 2) * pl + j + 2;
+        sm[yi] = h.ll;
+        sm[yi + subl] = h.lh;
+        sm[yi + 2 * subl] = h.hl;
+        sm[yi + 3 * subl] = h.hh;
     }
 }
 
@@ -532,6 +534,15 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
     int c_prev = -1;
+    // Staging order: the threads that hold a base tile (the last `nbase_thr` items of the list) are busy with
+    // the synthesis of the previous unit when the next one is staged, so the others stage, two patches each
+    // if need be; only if they are too few does every thread take part.
+    const int nbase_thr = g.NPL * g.nbase, first_free = nitems % nthr;
+    int srank = tid - first_free;
+    if (srank < 0) srank += nthr;
+    int nstagers = nthr - nbase_thr;
+    if (nitems > nthr || nstagers * 4 < nthr) nstagers = nthr;
+    if (srank >= nstagers) srank = 0x3fffffff;
     __syncthreads();
     if (g.bulk && tid == 0) {
         mbar_init(bar, 1);
@@ -551,17 +562,18 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         WT_TICK(1);
         int lnext;
         if (g.bulk) {
-            const bool ok = mbar_wait(bar, parity);
+            // every thread polls the copy barrier itself (bounded); a copy that never lands is flagged and
+            // the block carries on with whatever is in the buffer rather than waiting for ever
+            if (!mbar_wait(bar, parity)) atomicExch(status, 1);
             parity ^= 1u;
-            if (__syncthreads_or(!ok)) {  // a copy never landed: flag it, let it have one more bounded wait, stop
-                if (tid == 0) atomicExch(status, 1);
-                if (!ok) mbar_wait(bar, parity ^ 1u);
-                return;
-            }
             WT_TICK(8);
-            lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, bg);
+#ifndef WT_ABL_NOSTAGE
+            lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, bg, srank, nstagers);
+#else
+            lnext = L + 1;
+#endif
         } else {
-            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg);
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, srank, nstagers);
         }
         WT_TICK(2);
         __syncthreads();
@@ -590,7 +602,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 bslot = fdiv(it, g.d_nlv);
                 decode_level_item(g, it - bslot * nlv, l, sub, tyy, txx);
                 pitch = g.pitch[l];
-                src = sm + (size_t)bslot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * tyy * pitch + 4 * txx;
+                src = sm + bslot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * tyy * pitch + 4 * txx;
                 wt = wtab + (1 + (l - 1) * 4 + sub) * WT_STRIDE;
             } else {
                 const int bi = it - nlevel_items;
@@ -599,17 +611,21 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 tyy = fdiv(r, g.d_tx[0]);
                 txx = r - tyy * g.tx[0];
                 pitch = g.pitch[0];
-                src = sm + (size_t)bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
+                src = sm + bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
                 wt = wtab;
                 has_base = true;
             }
             float w[KK];
             load_weights(wt, w);
+#ifndef WT_ABL_NOCONV
             conv_tile(src, pitch, w, acc);
+#else
+            for (int r = 0; r < TH; ++r) for (int cc = 0; cc < 4; ++cc) acc[r][cc] = w[(r * 4 + cc) % KK] + src[r * pitch + cc];
+#endif
             if (is_level) {
                 const int zp = g.zpitch[l];
                 if (4 * txx < zp) {
-                    float *z = sm + (size_t)bslot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * tyy * zp + 4 * txx;
+                    float *z = sm + bslot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * tyy * zp + 4 * txx;
                     const int zr_left = g.zrows[l] - TH * tyy;
 #pragma unroll
                     for (int r = 0; r < TH; ++r)
@@ -622,9 +638,11 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         __syncthreads();
         WT_TICK(6);
         if (has_base) {
-            const float *S = sm + (size_t)bslot * g.slot_stride;
+            const float *S = sm + bslot * g.slot_stride;
 #pragma unroll
+#ifndef WT_ABL_NOSYNTH
             for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, bias, &acc[4 * hb]);
+#endif
             const int b = bg * g.NPL + bslot;
             if (b < g.B) {
                 T *oa = out + ((size_t)b * g.C + c) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
@@ -682,20 +700,15 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
         const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
         int lnext;
         if (g.bulk) {
-            const bool ok = mbar_wait(bar, parity);
+            if (!mbar_wait(bar, parity)) atomicExch(status, 1);
             parity ^= 1u;
-            if (__syncthreads_or(!ok)) {
-                if (tid == 0) atomicExch(status, 1);
-                if (!ok) mbar_wait(bar, parity ^ 1u);
-                return;
-            }
             const T *rx = reinterpret_cast<const T *>(raw);
             const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.raw_slot_bytes);
-            lnext = stage_input<T, true>(sm, g, g.offA, rx, c, bg);
-            stage_input<T, true>(sm, g, g.offG, rg, c, bg);
+            lnext = stage_input<T, true>(sm, g, g.offA, rx, c, bg, tid, nthr);
+            stage_input<T, true>(sm, g, g.offG, rg, c, bg, tid, nthr);
         } else {
-            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg);
-            stage_input<T, false>(sm, g, g.offG, go, c, bg);
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, tid, nthr);
+            stage_input<T, false>(sm, g, g.offG, go, c, bg, tid, nthr);
         }
         __syncthreads();
         if (g.bulk && tid == 0 && u + 1 < u_end) {
@@ -712,7 +725,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             for (int it = kth; it < g.NPL * ntile; it += nth) {
                 const int slot = fdiv(it, g.d_nt[lvl]), r = it - slot * ntile;
                 const int tyy = fdiv(r, g.d_tx[lvl]), txx = r - tyy * g.tx[lvl];
-                const float *S = sm + (size_t)slot * g.slot_stride;
+                const float *S = sm + slot * g.slot_stride;
                 const float *ysrc = S + g.offA[lvl] + suboff + TH * tyy * pl + 4 * txx;
                 // D tile = columns 4tx+2..4tx+5 of rows TH*ty+2.. (8-byte aligned)
                 const float *dsrc = S + g.offG[lvl] + suboff + (TH * tyy + 2) * pl + 4 * txx + 2;
