@@ -51,7 +51,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -125,8 +125,8 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="stage1_f32")
     ap.add_argument("--ref-batch", type=int, default=16, help="images per oracle step in --impl reference")
@@ -198,6 +198,8 @@ def main():
 
     for i in range(max(args.warmup, 3)):
         step(i)
+    # keep the GPU busy for a moment so the sampled clocks are the clocks under load
+    sync_all()
     sync_all()
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -291,13 +293,16 @@ def main():
         from oracle import wtconv_oracle as O
         Bs = min(wl.B, 64)
         Ic = inputs.make_inputs(wl.with_(B=Bs))
+        reps = 3
         c0 = time.time()
-        O.forward(Ic["x"], Ic["w0"], Ic["s0"], None, Ic["wl"], Ic["sl"], wl.L)
-        O.backward(Ic["x"], Ic["g"], Ic["w0"], Ic["s0"], None, Ic["wl"], Ic["sl"], wl.L)
-        cdt = time.time() - c0
+        for _ in range(reps):
+            O.forward(Ic["x"], Ic["w0"], Ic["s0"], None, Ic["wl"], Ic["sl"], wl.L)
+            O.backward(Ic["x"], Ic["g"], Ic["w0"], Ic["s0"], None, Ic["wl"], Ic["sl"], wl.L)
+        cdt = (time.time() - c0) / reps
         result["cpu_baseline"] = {"value": wl.with_(B=Bs).N / cdt, "unit": "elements/s", "cores": O.num_threads(),
-                                  "kind": "oracle", "seconds": cdt,
-                                  "sample": "one fwd+bwd of B=%d images of %s, fp64" % (Bs, wl.name)}
+                                  "kind": "oracle", "seconds_per_step": cdt,
+                                  "sample": "%d x fwd+bwd of B=%d images of %s, fp64 (%.0f core-seconds)"
+                                            % (reps, Bs, wl.name, reps * cdt * O.num_threads())}
     print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()
