@@ -128,6 +128,33 @@ wtconv_status wtconv_backward(const wtconv_desc *desc, const void *x, const void
                               float *grad_wl, float *grad_sl,
                               void *workspace, size_t workspace_bytes, void *stream);
 
+/* Backward pass for callers that cannot hand over a workspace.  (The paper has no counterpart: it never
+ * discusses where its kernels' scratch comes from.)
+ *
+ * Some hosts of this library may not allocate device memory at the point where they call the backward pass:
+ * an inference or training runtime that froze its memory plan at start-up, a plug-in that is only given the
+ * input and output buffers, or a latency-critical loop in which cudaMalloc (which may synchronise the device
+ * and can fail once memory is fragmented) is off limits.  This variant of wtconv_backward needs no workspace
+ * argument: its scratch is a WTCONV_STATIC_SCRATCH_BYTES array built into the library image (so each GPU that
+ * loads the library carries that much memory until the process exits).  It calls no cudaMalloc, cudaFree or
+ * any other allocating routine.
+ *
+ * Same arguments, layouts, outputs and arithmetic as wtconv_backward, minus the workspace.  Differences:
+ *   - WTCONV_ERR_WORKSPACE is returned, before anything is launched, when the descriptor needs more scratch
+ *     than the built-in array holds (wtconv_workspace_bytes tells how much a descriptor needs; the shapes the
+ *     whole-plane kernels serve need well under 1 MiB, large planes on the tiled path need far more).
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device current); make that first call outside any stream capture.  Later calls on that device reuse it.
+ *   - All calls on one device share the one array, and it keeps whatever the last call left in it.  Each call
+ *     clears what has to start at zero, so stale contents are harmless, but two calls whose kernels overlap
+ *     on the GPU (different streams) race on it: serialise them, or use wtconv_backward with two workspaces. */
+#define WTCONV_STATIC_SCRATCH_BYTES (8u << 20)
+wtconv_status wtconv_backward_static(const wtconv_desc *desc, const void *x, const void *grad_out,
+                                     const float *w0, const float *s0, const float *b0,
+                                     const float *wl, const float *sl,
+                                     void *grad_x, float *grad_w0, float *grad_s0, float *grad_b0,
+                                     float *grad_wl, float *grad_sl, void *stream);
+
 /* One training step from HOST memory: copies x, grad_out and the parameters to the device,
  * runs wtconv_forward and wtconv_backward, and copies out, grad_x and the parameter
  * gradients back, all asynchronously on `stream` (the host buffers should be pinned for the

@@ -6,6 +6,8 @@
 #include "tiled_kernels.cuh"
 #include "plane_kernels.cuh"
 
+#include <mutex>
+
 namespace {
 
 using wt::host_half_up;
@@ -263,6 +265,31 @@ ParamSizes param_sizes(const wtconv_desc *d) {
     return {C * KK * 4, C * 4, L * C * 4 * KK * 4, L * C * 4 * 4};
 }
 
+// ------------------------------------------------------------------ allocation-free backward
+// Scratch for wtconv_backward_static: lives in the library image, so every GPU that loads the library holds
+// these bytes until the process exits.  Its name is only a host-side handle; the device address is looked
+// up once per device with cudaGetSymbolAddress (see static_scratch_for_current_device).
+static __device__ __align__(256) unsigned char wt_static_scratch[WTCONV_STATIC_SCRATCH_BYTES];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_scratch_mutex;
+void *g_scratch_ptr[MAX_DEVICES] = {};
+
+// Device address of wt_static_scratch on the current device; resolved on the first call per device.
+wtconv_status static_scratch_for_current_device(void **out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WTCONV_ERR_CUDA;
+    if (dev < 0 || dev >= MAX_DEVICES) return WTCONV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, wt_static_scratch) != cudaSuccess || !p) return WTCONV_ERR_CUDA;
+        g_scratch_ptr[dev] = p;
+    }
+    *out = g_scratch_ptr[dev];
+    return WTCONV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -429,6 +456,21 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     d2h(h_gwl, gwl, ps.wl);
     d2h(h_gsl, gsl, ps.sl);
     return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
+}
+
+wtconv_status wtconv_backward_static(const wtconv_desc *d, const void *x, const void *grad_out, const float *w0,
+                                     const float *s0, const float *b0, const float *wl, const float *sl, void *grad_x,
+                                     float *grad_w0, float *grad_s0, float *grad_b0, float *grad_wl, float *grad_sl,
+                                     void *stream) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (bwd_ws_bytes(d) > (size_t)WTCONV_STATIC_SCRATCH_BYTES) return WTCONV_ERR_WORKSPACE;  // shape needs more scratch than is built in
+    void *scratch = nullptr;
+    if ((st = static_scratch_for_current_device(&scratch)) != WTCONV_OK) return st;
+    // wtconv_backward clears the parts of its workspace that must start at zero on every call, so the
+    // contents a previous call left in the shared array do not matter.
+    return wtconv_backward(d, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad_s0, grad_b0, grad_wl, grad_sl,
+                           scratch, (size_t)WTCONV_STATIC_SCRATCH_BYTES, stream);
 }
 
 #ifdef WT_PHASE_TIMING

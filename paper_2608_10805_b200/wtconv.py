@@ -19,8 +19,8 @@ _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_NAMES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
 
 EXPORTS = ["wtconv_status_string", "wtconv_level_shape", "wtconv_workspace_bytes", "wtconv_plan_name",
-           "wtconv_launch_count", "wtconv_forward", "wtconv_backward", "wtconv_step_host_workspace_bytes",
-           "wtconv_step_host"]
+           "wtconv_launch_count", "wtconv_forward", "wtconv_backward", "wtconv_backward_static",
+           "wtconv_step_host_workspace_bytes", "wtconv_step_host"]
 
 
 class Desc(ctypes.Structure):
@@ -55,6 +55,7 @@ def lib():
         L.wtconv_launch_count.argtypes = [dp, i32p, i32p]
         L.wtconv_forward.argtypes = [dp] + [vp] * 7 + [vp, sz, vp]
         L.wtconv_backward.argtypes = [dp] + [vp] * 13 + [vp, sz, vp]
+        L.wtconv_backward_static.argtypes = [dp] + [vp] * 13 + [vp]
         L.wtconv_step_host_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz)]
         L.wtconv_step_host.argtypes = [dp] + [vp] * 14 + [vp, sz, vp]
         _lib = L
@@ -125,6 +126,19 @@ def wtconv_backward(desc, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad
     _check(lib().wtconv_backward(ctypes.byref(desc), _ptr(x), _ptr(grad_out), _ptr(w0), _ptr(s0), _ptr(b0), _ptr(wl),
                                  _ptr(sl), _ptr(grad_x), _ptr(grad_w0), _ptr(grad_s0), _ptr(grad_b0), _ptr(grad_wl),
                                  _ptr(grad_sl), _ptr(workspace), workspace.numel(), _stream(stream)))
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def wtconv_backward_static(desc, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad_s0, grad_b0, grad_wl, grad_sl,
+                           stream=None):
+    """wtconv_backward without a workspace argument, for callers that must not allocate device memory:
+    the scratch is an array built into the library (see include/wtconv.h for its limits)."""
+    _need_cuda(x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad_s0, grad_b0, grad_wl, grad_sl)
+    _check(lib().wtconv_backward_static(ctypes.byref(desc), _ptr(x), _ptr(grad_out), _ptr(w0), _ptr(s0), _ptr(b0),
+                                        _ptr(wl), _ptr(sl), _ptr(grad_x), _ptr(grad_w0), _ptr(grad_s0), _ptr(grad_b0),
+                                        _ptr(grad_wl), _ptr(grad_sl), _stream(stream)))
 
 
 def wtconv_step_host_workspace_bytes(desc):
