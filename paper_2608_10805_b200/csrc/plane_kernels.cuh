@@ -537,12 +537,10 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     // Staging order: the threads that hold a base tile (the last `nbase_thr` items of the list) are busy with
     // the synthesis of the previous unit when the next one is staged, so the others stage, two patches each
     // if need be; only if they are too few does every thread take part.
-    const int nbase_thr = g.NPL * g.nbase, first_free = nitems % nthr;
-    int srank = tid - first_free;
-    if (srank < 0) srank += nthr;
-    int nstagers = nthr - nbase_thr;
-    if (nitems > nthr || nstagers * 4 < nthr) nstagers = nthr;
-    if (srank >= nstagers) srank = 0x3fffffff;
+    // whole warps that hold level tiles only (threads below the first base tile, rounded down to a warp)
+    int nstagers = nitems <= nthr ? (nlevel_items / 32) * 32 : nthr;
+    if (nstagers * 4 < nthr) nstagers = nthr;
+    const int srank = tid < nstagers ? tid : 0x3fffffff;
     __syncthreads();
     if (g.bulk && tid == 0) {
         mbar_init(bar, 1);
