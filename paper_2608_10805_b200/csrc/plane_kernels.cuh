@@ -206,6 +206,120 @@ __device__ __forceinline__ void ld4(const T *p, float (&v)[4]) {
     if (RAW) load4s(p, v); else load4(p, v);
 }
 
+__device__ __forceinline__ void decode_level_item(const Geom &g, int r, int &l, int &sub, int &tyy, int &txx);
+
+// ---- per-thread work descriptors.  A thread's tiles and staging patches are the same for every unit, so
+// ---- they are decoded once, before the unit loop, and live in registers.
+struct PatchD {   // 4x4 pixel staging patch (vector path, L >= 2)
+    int so;       // element offset of the patch inside its plane: y*W + 4q
+    int xi, yi, y2;  // float indices of its first x / level-1 / level-2 element in shared memory
+    int meta;     // bit 31 valid, bits 0-7 plane slot, bits 8-10 rows inside the image (1..4)
+};
+__device__ __forceinline__ PatchD decode_patch(const Geom &g, const int *off, int e) {
+    PatchD p;
+    p.meta = 0;
+    p.so = p.xi = p.yi = p.y2 = 0;
+    if (e < g.NPL * g.npatch4) {
+        const int slot = fdiv(e, g.d_npatch4), r = e - slot * g.npatch4;
+        const int i2 = fdiv(r, g.d_prow), q = r - i2 * (int)g.d_prow.d;
+        const int y = 4 * i2, S = slot * g.slot_stride;
+        int nrows = g.H - y;
+        if (nrows > 4) nrows = 4;
+        p.so = y * g.W + 4 * q;
+        p.xi = S + off[0] + (y + 2) * g.pitch[0] + 4 * q + 2;
+        p.yi = S + off[1] + (2 * i2 + 2) * g.pitch[1] + 2 * q + 2;
+        p.y2 = S + off[2] + (i2 + 2) * g.pitch[2] + q + 2;
+        p.meta = (int)(0x80000000u | (unsigned)slot | ((unsigned)nrows << 8));
+    }
+    return p;
+}
+template <typename T, bool RAW>
+__device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD &p, const T *__restrict__ gsrc,
+                                          int img_stride, int bg) {
+    if (p.meta >= 0) return;
+    const int slot = p.meta & 0xff, nrows = (p.meta >> 8) & 7;
+    const int p0 = g.pitch[0], p1 = g.pitch[1], sub1 = g.rows[1] * p1, sub2 = g.rows[2] * g.pitch[2], W = g.W;
+    float a[4][4];
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) a[rr][cc] = 0.f;
+    if (bg * g.NPL + slot < g.B) {
+        const T *pa = gsrc + (size_t)slot * img_stride + p.so;
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr)
+            if (rr < nrows) ld4<T, RAW>(pa + rr * W, a[rr]);
+    }
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+        if (rr < nrows) {
+            *reinterpret_cast<float2 *>(&sm[p.xi + rr * p0]) = make_float2(a[rr][0], a[rr][1]);
+            *reinterpret_cast<float2 *>(&sm[p.xi + rr * p0 + 2]) = make_float2(a[rr][2], a[rr][3]);
+        }
+    }
+    Haar4 h[2][2];
+#pragma unroll
+    for (int bi = 0; bi < 2; ++bi)
+#pragma unroll
+        for (int bj = 0; bj < 2; ++bj)
+            h[bi][bj] = haar_butterfly(a[2 * bi][2 * bj], a[2 * bi][2 * bj + 1], a[2 * bi + 1][2 * bj], a[2 * bi + 1][2 * bj + 1]);
+#pragma unroll
+    for (int bi = 0; bi < 2; ++bi) {
+        *reinterpret_cast<float2 *>(&sm[p.yi + bi * p1]) = make_float2(h[bi][0].ll, h[bi][1].ll);
+        *reinterpret_cast<float2 *>(&sm[p.yi + bi * p1 + sub1]) = make_float2(h[bi][0].lh, h[bi][1].lh);
+        *reinterpret_cast<float2 *>(&sm[p.yi + bi * p1 + 2 * sub1]) = make_float2(h[bi][0].hl, h[bi][1].hl);
+        *reinterpret_cast<float2 *>(&sm[p.yi + bi * p1 + 3 * sub1]) = make_float2(h[bi][0].hh, h[bi][1].hh);
+    }
+    const Haar4 h2 = haar_butterfly(h[0][0].ll, h[0][1].ll, h[1][0].ll, h[1][1].ll);
+    sm[p.y2] = h2.ll;
+    sm[p.y2 + sub2] = h2.lh;
+    sm[p.y2 + 2 * sub2] = h2.hl;
+    sm[p.y2 + 3 * sub2] = h2.hh;
+}
+
+struct ItemD {    // one 4 x TH conv tile
+    int src;      // float index of the window's top-left element
+    int wt;       // float index of its 25 folded weights
+    int z;        // level tile: float index of its output in Z^l, or -2 if the tile lies outside what the synthesis reads;
+                  // base tile: -1
+    int meta;     // bit 31 valid; bits 0-9 window pitch; bits 10-19 Z pitch; bits 20-23 rows to store (0..TH)
+};
+__device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_items, int nitems, int &bslot, int &tyy,
+                                             int &txx, bool &is_base) {
+    ItemD d;
+    d.src = d.wt = 0;
+    d.z = -2;
+    d.meta = 0;
+    if (it >= nitems) return d;
+    const int nlv = g.lvl_start[g.L + 1];
+    if (it < nlevel_items) {
+        int l, sub, ty2, tx2;
+        const int slot = fdiv(it, g.d_nlv);
+        decode_level_item(g, it - slot * nlv, l, sub, ty2, tx2);
+        const int pitch = g.pitch[l], zp = g.zpitch[l];
+        d.src = slot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * ty2 * pitch + 4 * tx2;
+        d.wt = g.wtab_off + (1 + (l - 1) * 4 + sub) * WT_STRIDE;
+        int zleft = g.zrows[l] - TH * ty2;
+        if (zleft > TH) zleft = TH;
+        if (4 * tx2 < zp && zleft > 0) d.z = slot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * ty2 * zp + 4 * tx2;
+        if (zleft < 0) zleft = 0;
+        d.meta = (int)(0x80000000u | (unsigned)pitch | ((unsigned)zp << 10) | ((unsigned)zleft << 20));
+    } else {
+        const int bi = it - nlevel_items;
+        bslot = fdiv(bi, g.d_nbase);
+        const int r = bi - bslot * g.nbase;
+        tyy = fdiv(r, g.d_tx[0]);
+        txx = r - tyy * g.tx[0];
+        const int pitch = g.pitch[0];
+        d.src = bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
+        d.wt = g.wtab_off;
+        d.z = -1;
+        d.meta = (int)(0x80000000u | (unsigned)pitch);
+        is_base = true;
+    }
+    return d;
+}
+
 // Stage the planes of one unit (channel c, images bg*NPL ..): x into the haloed array `off[0]`, its
 // level-1 Haar subbands (Eq. 5) into `off[1]` and, on the vector path with L >= 2, the level-2 subbands
 // into `off[2]` in the same pass (returns the first level that still has to be staged).  RAW = true reads
@@ -537,10 +651,24 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     // Staging order: the threads that hold a base tile (the last `nbase_thr` items of the list) are busy with
     // the synthesis of the previous unit when the next one is staged, so the others stage, two patches each
     // if need be; only if they are too few does every thread take part.
-    // whole warps that hold level tiles only (threads below the first base tile, rounded down to a warp)
-    int nstagers = nitems <= nthr ? (nlevel_items / 32) * 32 : nthr;
+    // Staging is done by whole warps that hold level tiles only (threads below the first base tile, rounded
+    // down to a warp) while the others run the previous unit's synthesis; if those are too few, by everybody.
+    int nstagers = (nlevel_items / 32) * 32;
+    if (nstagers > nthr) nstagers = nthr;
     if (nstagers * 4 < nthr) nstagers = nthr;
     const int srank = tid < nstagers ? tid : 0x3fffffff;
+    // hoisted descriptors: two tiles and two staging patches per thread cover the plans in use
+    constexpr int MAXI = 2;
+    const bool hoist_items = nitems <= MAXI * nthr;
+    const bool hoist_patch = g.vec && L >= 2 && g.NPL * g.npatch4 <= 2 * nstagers;
+    ItemD items[MAXI];
+    int bslot = 0, tyy = 0, txx = 0;
+    bool has_base = false;
+#pragma unroll
+    for (int k = 0; k < MAXI; ++k)
+        items[k] = decode_item(g, hoist_items ? tid + k * nthr : 0x3fffffff, nlevel_items, nitems, bslot, tyy, txx, has_base);
+    PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
+    PatchD patch1 = decode_patch(g, g.offA, hoist_patch && srank < nstagers ? srank + nstagers : 0x3fffffff);
     __syncthreads();
     if (g.bulk && tid == 0) {
         mbar_init(bar, 1);
@@ -565,11 +693,18 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             if (!mbar_wait(bar, parity)) atomicExch(status, 1);
             parity ^= 1u;
             WT_TICK(8);
-#ifndef WT_ABL_NOSTAGE
-            lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, bg, srank, nstagers);
-#else
-            lnext = L + 1;
-#endif
+            if (hoist_patch) {
+                run_patch<T, true>(sm, g, patch0, reinterpret_cast<const T *>(raw), g.raw_slot_bytes / (int)sizeof(T), bg);
+                run_patch<T, true>(sm, g, patch1, reinterpret_cast<const T *>(raw), g.raw_slot_bytes / (int)sizeof(T), bg);
+                lnext = 3;
+            } else {
+                lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, bg, srank, nstagers);
+            }
+        } else if (hoist_patch) {
+            const T *gsrc = x + ((size_t)bg * g.NPL * g.C + c) * HW;
+            run_patch<T, false>(sm, g, patch0, gsrc, g.C * (int)HW, bg);
+            run_patch<T, false>(sm, g, patch1, gsrc, g.C * (int)HW, bg);
+            lnext = 3;
         } else {
             lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, srank, nstagers);
         }
@@ -589,45 +724,37 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         // ---- one item list: level tiles (Z^l = Wfold^l (*) Y^l) first, base tiles last; a thread's last
         //      item may be a base tile, which stays in registers across the barrier
         float acc[TH][4];
-        int bslot = 0, tyy = 0, txx = 0;
-        bool has_base = false;
-        for (int it = tid; it < nitems; it += nthr) {
-            const float *src;
-            const float *wt;
-            int pitch, l = 0, sub = 0;
-            const bool is_level = it < nlevel_items;
-            if (is_level) {
-                bslot = fdiv(it, g.d_nlv);
-                decode_level_item(g, it - bslot * nlv, l, sub, tyy, txx);
-                pitch = g.pitch[l];
-                src = sm + bslot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * tyy * pitch + 4 * txx;
-                wt = wtab + (1 + (l - 1) * 4 + sub) * WT_STRIDE;
-            } else {
-                const int bi = it - nlevel_items;
-                bslot = fdiv(bi, g.d_nbase);
-                const int r = bi - bslot * g.nbase;
-                tyy = fdiv(r, g.d_tx[0]);
-                txx = r - tyy * g.tx[0];
-                pitch = g.pitch[0];
-                src = sm + bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
-                wt = wtab;
-                has_base = true;
+        if (hoist_items) {
+#pragma unroll
+            for (int k = 0; k < MAXI; ++k) {
+                if (items[k].meta < 0) {
+                    float w[KK];
+                    load_weights(sm + items[k].wt, w);
+                    conv_tile(sm + items[k].src, items[k].meta & 0x3ff, w, acc);
+                    if (items[k].z >= 0) {
+                        const int zp = (items[k].meta >> 10) & 0x3ff, zleft = (items[k].meta >> 20) & 0xf;
+                        float *z = sm + items[k].z;
+#pragma unroll
+                        for (int r = 0; r < TH; ++r)
+                            if (r < zleft) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+                    }
+                }
             }
-            float w[KK];
-            load_weights(wt, w);
-#ifndef WT_ABL_NOCONV
-            conv_tile(src, pitch, w, acc);
-#else
-            for (int r = 0; r < TH; ++r) for (int cc = 0; cc < 4; ++cc) acc[r][cc] = w[(r * 4 + cc) % KK] + src[r * pitch + cc];
-#endif
-            if (is_level) {
-                const int zp = g.zpitch[l];
-                if (4 * txx < zp) {
-                    float *z = sm + bslot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * tyy * zp + 4 * txx;
-                    const int zr_left = g.zrows[l] - TH * tyy;
+        } else {
+            has_base = false;
+            for (int it = tid; it < nitems; it += nthr) {
+                bool isb = false;
+                const ItemD d = decode_item(g, it, nlevel_items, nitems, bslot, tyy, txx, isb);
+                has_base = isb;
+                float w[KK];
+                load_weights(sm + d.wt, w);
+                conv_tile(sm + d.src, d.meta & 0x3ff, w, acc);
+                if (d.z >= 0) {
+                    const int zp = (d.meta >> 10) & 0x3ff, zleft = (d.meta >> 20) & 0xf;
+                    float *z = sm + d.z;
 #pragma unroll
                     for (int r = 0; r < TH; ++r)
-                        if (r < zr_left) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+                        if (r < zleft) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
                 }
             }
         }
@@ -899,11 +1026,12 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
                 int nblocks = NUM_SMS * bps;
                 if (nblocks > units) nblocks = units;
                 // thread-slot use x resident warps (about 16 hide the latency-bound phases) x phase overlap
-                double occ = (double)bps * T / 512.0;
+                double occ = (double)bps * T / 384.0;
                 if (occ > 1.0) occ = 1.0;
                 const double overlap = bps >= 4 ? 1.0 : (bps == 3 ? 0.95 : (bps == 2 ? 0.8 : 0.55));
-                const double sc = eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) *
-                                  partition_eff(units, nblocks) * ((double)B / ((double)bgroups * npl));
+                const double sc = eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) * (rounds <= 2 ? 1.0 : 0.9) *
+                                  partition_eff(units, nblocks) * ((double)B / ((double)bgroups * npl)) *
+                                  (1.0 - 1e-4 * T / 32.0);
                 if (sc > best.score + 1e-9) {
                     best = cg;
                     best.smem_floats = (int)smem_floats; best.bgroups = bgroups; best.units = units;
@@ -1023,7 +1151,9 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
         if (e != cudaSuccess) return e;                                                             \
         kern<<<g.nblocks, g.nthreads, smem, st>>>(g, x, w0, s0, b0, wl, sl, out, status);           \
     }
-    if (g.nthreads * g.blocks_per_sm <= 512) {
+    if (g.nthreads <= 128 && g.blocks_per_sm <= 3) {
+        WT_LAUNCH_FWD(128, 3)
+    } else if (g.nthreads * g.blocks_per_sm <= 512) {
         if (g.nthreads <= 128) WT_LAUNCH_FWD(128, 4) else WT_LAUNCH_FWD(256, 2)
     } else {
         if (g.nthreads <= 128) WT_LAUNCH_FWD(128, 6) else WT_LAUNCH_FWD(256, 3)
