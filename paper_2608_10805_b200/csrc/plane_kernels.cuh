@@ -234,9 +234,13 @@ __device__ __forceinline__ PatchD decode_patch(const Geom &g, const int *off, in
     return p;
 }
 template <typename T, bool RAW>
-__device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD &p, const T *__restrict__ gsrc,
-                                          int img_stride, int bg) {
-    if (p.meta >= 0) return;
+__device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD &p0_, const T *__restrict__ gsrc,
+                                          int img_stride, int bg, int d0 = 0, int d1 = 0, int d2 = 0) {
+    if (p0_.meta >= 0) return;
+    PatchD p = p0_;  // d0/d1/d2 shift the x / level-1 / level-2 targets to another set of arrays (grad_out side)
+    p.xi += d0;
+    p.yi += d1;
+    p.y2 += d2;
     const int slot = p.meta & 0xff, nrows = (p.meta >> 8) & 7;
     const int p0 = g.pitch[0], p1 = g.pitch[1], sub1 = g.rows[1] * p1, sub2 = g.rows[2] * g.pitch[2], W = g.W;
     float a[4][4];
@@ -282,12 +286,14 @@ struct ItemD {    // one 4 x TH conv tile
     int wt;       // float index of its 25 folded weights
     int z;        // level tile: float index of its output in Z^l, or -2 if the tile lies outside what the synthesis reads;
                   // base tile: -1
-    int meta;     // bit 31 valid; bits 0-9 window pitch; bits 10-19 Z pitch; bits 20-23 rows to store (0..TH)
+    int meta;     // bit 31 valid; bits 0-9 window pitch; bits 10-19 Z pitch; bits 20-23 rows to store (0..TH);
+                  // bits 24-29 parameter class (0 = base, 1 + 4(l-1) + sub = level l subband sub)
+    int dg;       // float offset from this tile's x-side array to the matching grad_out-side array (backward kernel)
 };
 __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_items, int nitems, int &bslot, int &tyy,
                                              int &txx, bool &is_base) {
     ItemD d;
-    d.src = d.wt = 0;
+    d.src = d.wt = d.dg = 0;
     d.z = -2;
     d.meta = 0;
     if (it >= nitems) return d;
@@ -303,7 +309,9 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         if (zleft > TH) zleft = TH;
         if (4 * tx2 < zp && zleft > 0) d.z = slot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * ty2 * zp + 4 * tx2;
         if (zleft < 0) zleft = 0;
-        d.meta = (int)(0x80000000u | (unsigned)pitch | ((unsigned)zp << 10) | ((unsigned)zleft << 20));
+        d.meta = (int)(0x80000000u | (unsigned)pitch | ((unsigned)zp << 10) | ((unsigned)zleft << 20) |
+                       ((unsigned)(1 + (l - 1) * 4 + sub) << 24));
+        d.dg = g.offG[l] - g.offA[l];
     } else {
         const int bi = it - nlevel_items;
         bslot = fdiv(bi, g.d_nbase);
@@ -315,6 +323,7 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         d.wt = g.wtab_off;
         d.z = -1;
         d.meta = (int)(0x80000000u | (unsigned)pitch);
+        d.dg = g.offG[0] - g.offA[0];
         is_base = true;
     }
     return d;
@@ -918,6 +927,166 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     }
 }
 
+// ------------------------------------------------------------------ fused backward kernel
+// One pass over x and grad_out gives grad_x and the weight-gradient partial sums.  Both decompositions are
+// staged (x -> X, Y^l; grad_out -> G, D^l).  Each thread owns exactly one tile of the item list (so its
+// parameter class never changes) and does two things with it:
+//   weight gradient  dWfold[u,v] += sum_tile D[i,j] * Y[i+u-2, j+v-2]          (Sec. 2.2; 25 register accumulators
+//                                                                              that live across all images of a channel)
+//   input gradient   the forward dataflow on grad_out with rotated kernels: conv of the D window, then the
+//                    closed-form synthesis of Proposition 2 and the store of grad_x.
+// Used when a unit's item list fits one round of the block (<= 256 tiles); otherwise the separate weight-
+// gradient and input-gradient kernels run.
+template <typename T>
+__global__ void __launch_bounds__(256, 2)
+plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
+                 const float *__restrict__ w0, const float *__restrict__ s0, const float *__restrict__ wl,
+                 const float *__restrict__ sl, T *__restrict__ gx, float *__restrict__ part0,
+                 float *__restrict__ partl /* level l at l*C*np*100 */) {
+    extern __shared__ __align__(16) float sm[];
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
+    float *wtab = sm + g.wtab_off;
+    const int L = g.L, nlv = g.lvl_start[L + 1], ncls = 1 + 4 * L;
+    const int nlevel_items = g.NPL * nlv, nitems = nlevel_items + g.NPL * g.nbase;
+    const size_t HW = (size_t)g.H * g.W;
+    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
+    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
+    int bslot = 0, tyy = 0, txx = 0;
+    bool has_base = false;
+    const ItemD item = decode_item(g, tid, nlevel_items, nitems, bslot, tyy, txx, has_base);
+    const int cls = (item.meta >> 24) & 0x3f;
+    const bool hoist_patch = g.vec && L >= 2 && g.NPL * g.npatch4 <= 2 * nthr;
+    const PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? tid : 0x3fffffff);
+    const PatchD patch1 = decode_patch(g, g.offA, hoist_patch ? tid + nthr : 0x3fffffff);
+    const int dA0 = g.offG[0] - g.offA[0], dA1 = L >= 1 ? g.offG[1] - g.offA[1] : 0, dA2 = L >= 2 ? g.offG[2] - g.offA[2] : 0;
+    float accw[KK], gsum = 0.f;
+#pragma unroll
+    for (int t = 0; t < KK; ++t) accw[t] = 0.f;
+    int c_prev = -1;
+    __syncthreads();
+    for (int u = u_begin; u < u_end; ++u) {
+        const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
+        if (c != c_prev) {
+            build_weight_table(wtab, g, c, true, w0, s0, nullptr, wl, sl);
+            c_prev = c;
+        }
+        int lnext;
+        if (hoist_patch) {
+            const size_t po = ((size_t)bg * g.NPL * g.C + c) * HW;
+            run_patch<T, false>(sm, g, patch0, x + po, g.C * (int)HW, bg);
+            run_patch<T, false>(sm, g, patch0, go + po, g.C * (int)HW, bg, dA0, dA1, dA2);
+            run_patch<T, false>(sm, g, patch1, x + po, g.C * (int)HW, bg);
+            run_patch<T, false>(sm, g, patch1, go + po, g.C * (int)HW, bg, dA0, dA1, dA2);
+            lnext = 3;
+        } else {
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, tid, nthr);
+            stage_input<T, false>(sm, g, g.offG, go, c, bg, tid, nthr);
+        }
+        __syncthreads();
+        for (int l = lnext; l <= L; ++l) {
+            stage_level(sm, g, g.offA, l);
+            stage_level(sm, g, g.offG, l);
+            __syncthreads();
+        }
+        float acc[TH][4];
+        if (item.meta < 0) {
+            const int pitch = item.meta & 0x3ff;
+            const float *ysrc = sm + item.src;            // Y window (x side)
+            const float *gsrc = sm + item.src + item.dg;  // D window (grad_out side)
+            {
+                // weight gradient: the tile's D values are the window's interior
+                float d[TH][4];
+#pragma unroll
+                for (int rr = 0; rr < TH; ++rr) {
+                    const float2 q0 = *reinterpret_cast<const float2 *>(gsrc + (rr + 2) * pitch + 2);
+                    const float2 q1 = *reinterpret_cast<const float2 *>(gsrc + (rr + 2) * pitch + 4);
+                    d[rr][0] = q0.x; d[rr][1] = q0.y; d[rr][2] = q1.x; d[rr][3] = q1.y;
+                }
+                if (cls == 0) {
+#pragma unroll
+                    for (int rr = 0; rr < TH; ++rr)
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) gsum += d[rr][cc];
+                }
+#pragma unroll
+                for (int rr = 0; rr < TH + 4; ++rr) {
+                    const float4 q0 = *reinterpret_cast<const float4 *>(ysrc + rr * pitch);
+                    const float4 q1 = *reinterpret_cast<const float4 *>(ysrc + rr * pitch + 4);
+                    const float in[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+                    for (int uu = 0; uu < 5; ++uu) {
+                        const int dr = rr - uu;
+                        if (dr >= 0 && dr < TH) {
+#pragma unroll
+                            for (int v = 0; v < 5; ++v)
+#pragma unroll
+                                for (int cc = 0; cc < 4; ++cc) accw[uu * 5 + v] = fmaf(d[dr][cc], in[cc + v], accw[uu * 5 + v]);
+                        }
+                    }
+                }
+            }
+            // input gradient: rotated-kernel conv of the D window
+            float w[KK];
+            load_weights(sm + item.wt, w);
+            conv_tile(gsrc, pitch, w, acc);
+            if (item.z >= 0) {
+                const int zp = (item.meta >> 10) & 0x3ff, zleft = (item.meta >> 20) & 0xf;
+                float *z = sm + item.z;
+#pragma unroll
+                for (int r = 0; r < TH; ++r)
+                    if (r < zleft) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
+            }
+        }
+        __syncthreads();
+        if (has_base) {
+            const float *S = sm + bslot * g.slot_stride;
+#pragma unroll
+            for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, 0.f, &acc[4 * hb]);
+            const int b = bg * g.NPL + bslot;
+            if (b < g.B) {
+                T *oa = gx + ((size_t)b * g.C + c) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
+                const bool vec = g.vec && (4 * txx + 3 < g.W);
+#pragma unroll
+                for (int r = 0; r < TH; ++r)
+                    if (TH * tyy + r < g.H) store_row4(oa + (size_t)r * g.W, 4 * txx, g.W, vec, acc[r]);
+            }
+        }
+        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_bg) != c);
+        if (last_of_channel) {
+            // block tree through shared memory: park the 26 sums and the class of every thread in the array
+            // region (idle now), then one thread per (class, tap) adds its class's threads in index order
+            __syncthreads();
+            float *scr = sm;
+#pragma unroll
+            for (int t = 0; t < KK; ++t) scr[tid * (KK + 2) + t] = accw[t];
+            scr[tid * (KK + 2) + KK] = gsum;
+            scr[tid * (KK + 2) + KK + 1] = __int_as_float(item.meta < 0 ? cls : -1);
+            __syncthreads();
+            const int slotp = blockIdx.x - block_of_unit((long long)c * g.bgroups, gridDim.x, g.units);
+            for (int e = tid; e < ncls * (KK + 1); e += nthr) {
+                const int c2 = e / (KK + 1), t = e - c2 * (KK + 1);
+                if (c2 > 0 && t == KK) continue;
+                float sacc = 0.f;
+                for (int th = 0; th < nthr; ++th)
+                    if (__float_as_int(scr[th * (KK + 2) + KK + 1]) == c2) sacc += scr[th * (KK + 2) + t];
+                if (c2 == 0) {
+                    part0[((size_t)c * g.np + slotp) * (KK + 1) + t] = sacc;
+                } else {
+                    const int l = (c2 - 1) >> 2, sb_ = (c2 - 1) & 3;
+                    partl[(size_t)l * g.C * g.np * 4 * KK + (((size_t)c * g.np + slotp) * 4 + sb_) * KK + t] = sacc;
+                }
+            }
+            __syncthreads();
+            for (int i = tid; i < g.wtab_off; i += nthr) sm[i] = 0.f;  // restore the zero halos of the arrays
+#pragma unroll
+            for (int t = 0; t < KK; ++t) accw[t] = 0.f;
+            gsum = 0.f;
+        }
+        __syncthreads();  // arrays and Z are free again for the next unit's staging
+    }
+}
+
 // ------------------------------------------------------------------ host-side planning
 inline void fill_common(Geom &g, int B, int C, int H, int W, int L, int elem_bytes) {
     g.B = B; g.C = C; g.H = H; g.W = W; g.L = L;
@@ -1121,6 +1290,62 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
     return found;
 }
 
+// Fused-backward plan: one round (every tile its own thread), both input pyramids plus Z in shared memory, no
+// bulk prefetch.  tune bits 14-19: planes per unit, bits 20-22: blocks per SM (shared with the weight-gradient plan).
+inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    const int fNpl = (tune >> 14) & 63, fBps = (tune >> 20) & 7;
+    if ((tune >> 24) & 1) return false;  // bit 24: never fuse
+    Geom g = {};
+    fill_common(g, B, C, H, W, L, elem_bytes);
+    const int slot = layout_slot(g, true, true);
+    const int M = g.lvl_start[L + 1] + g.nbase;
+    const int wtab = (1 + 4 * L) * WT_STRIDE;
+    bool found = false;
+    best.score = -1.0;
+    for (int npl = 1; npl <= 64; ++npl) {
+        if (npl > 1 && npl > B) break;
+        if (fNpl && npl != fNpl) continue;
+        if (npl * M > 256) break;
+        const int T = (npl * M + 31) & ~31;
+        Geom cg = g;
+        cg.NPL = npl; cg.slot_stride = slot; cg.bulk = 0;
+        long long arrays = (long long)npl * slot;
+        const long long scratch = (long long)T * (KK + 2);
+        if (scratch > arrays) arrays = scratch;
+        const long long smem_floats = finish_layout(cg, arrays, wtab, 0, false);
+        const long long bytes = smem_floats * 4;
+        if (bytes > SMEM_LIMIT) break;
+        for (int bps = 1; bps <= 4; ++bps) {
+            if (bps * T > 512) continue;  // 128 registers per thread
+            if (fBps && bps != fBps) continue;
+            if (bps * (bytes + 1024) > SMEM_PER_SM) continue;
+            const int bgroups = (B + npl - 1) / npl, units = C * bgroups;
+            int nblocks = NUM_SMS * bps;
+            if (nblocks > units) nblocks = units;
+            double occ = (double)bps * T / 512.0;
+            if (occ > 1.0) occ = 1.0;
+            const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
+            const double sc = ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * partition_eff(units, nblocks) *
+                              ((double)B / ((double)bgroups * npl));
+            if (sc > best.score + 1e-9) {
+                best = cg;
+                best.smem_floats = (int)smem_floats;
+                best.bgroups = bgroups; best.units = units; best.d_bg = make_fastdiv(bgroups);
+                best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
+                int np = 1;
+                for (int ch = 0; ch < C; ++ch) {
+                    const int first = block_of_unit((long long)ch * bgroups, nblocks, units);
+                    const int last = block_of_unit((long long)(ch + 1) * bgroups - 1, nblocks, units);
+                    if (last - first + 1 > np) np = last - first + 1;
+                }
+                best.np = np;
+                found = true;
+            }
+        }
+    }
+    return found;
+}
+
 inline int dtype_bytes(int dtype) { return dtype == 0 ? 4 : 2; }
 
 inline bool supported(int H, int W, int k, int L, int dtype) {
@@ -1135,7 +1360,7 @@ constexpr size_t STATUS_BYTES = 256;
 inline size_t forward_workspace_bytes(int, int, int, int, int) { return STATUS_BYTES; }
 inline size_t backward_workspace_bytes(int B, int C, int H, int W, int L, int elem_bytes, unsigned tune = 0) {
     Geom g;
-    if (!plan_wgrad(B, C, H, W, L, elem_bytes, g, tune)) return 0;
+    if (!plan_bwd_fused(B, C, H, W, L, elem_bytes, g, tune) && !plan_wgrad(B, C, H, W, L, elem_bytes, g, tune)) return 0;
     return STATUS_BYTES + sizeof(float) * ((size_t)C * g.np * (KK + 1) + (size_t)L * C * g.np * 4 * KK);
 }
 
@@ -1177,6 +1402,25 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
                      const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st,
                      unsigned tune = 0) {
     Geom gw, gf;
+    if (plan_bwd_fused(B, C, H, W, L, (int)sizeof(T), gw, tune)) {
+        float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
+        float *partl = part0 + (size_t)C * gw.np * (KK + 1);
+        const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
+        cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // partial slots no block writes must read as zero
+        if (e != cudaSuccess) return e;
+        auto kb = plane_bwd_kernel<T>;
+        e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+        if (e != cudaSuccess) return e;
+        kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        ep->part0 = part0;
+        ep->np0 = gw.np;
+        for (int l = 0; l < L; ++l) {
+            ep->partl[l] = partl + (size_t)l * C * gw.np * 4 * KK;
+            ep->npl[l] = gw.np;
+        }
+        return cudaSuccess;
+    }
     if (!plan_wgrad(B, C, H, W, L, (int)sizeof(T), gw, tune) || !plan_forward(B, C, H, W, L, (int)sizeof(T), gf, tune))
         return cudaErrorInvalidValue;
     int *status = reinterpret_cast<int *>(ws);

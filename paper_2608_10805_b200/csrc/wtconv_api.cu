@@ -340,7 +340,11 @@ wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *b
     if (st != WTCONV_OK) return st;
     if (use_plane_path(d)) {
         if (fwd) *fwd = 1;
-        if (bwd) *bwd = 3; /* weight-gradient, input-gradient, epilogue (plus one memset node) */
+        if (bwd) {
+            wt::plane::Geom gq;
+            /* fused backward + epilogue, or weight-gradient + input-gradient + epilogue (plus one memset node) */
+            *bwd = wt::plane::plan_bwd_fused(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), gq, d->flags >> 8) ? 2 : 3;
+        }
     } else {
         if (fwd) *fwd = d->L + 1;
         if (bwd) *bwd = d->L + 2;
