@@ -99,13 +99,14 @@ struct Geom {
     int zrows[MAXL + 1], zpitch[MAXL + 1]; // conv outputs Z^l (forward kernel only)
     int offZ[MAXL + 1];
     int slot_stride;                       // floats per plane slot
-    int NPL;                               // plane slots per work unit (images of one channel)
+    int NPL;                               // plane slots per work unit: NPL consecutive channels of one image (contiguous in memory)
     int tx[MAXL + 1], ty[MAXL + 1];        // 4 x TH tiles per level grid (index 0 = base)
     int lvl_start[MAXL + 2];               // per plane: first level-item of level l (1..L); [L+1] = count
     int nbase;                             // base tiles per plane
     int wtab_off;                          // offset of the folded weight table [(1+4L)][WT_STRIDE] (bias at [0][25])
     int smem_floats;
-    int bgroups, units;                    // work units = C channels x bgroups image groups (channel-major)
+    int ngroups, units;                    // work units = ngroups channel groups x B images, group-major (a block keeps a group's
+                                           // weights and gradient accumulators while it walks through the images)
     int nthreads, nblocks, blocks_per_sm;
     int vec;                               // 1: W % 4 == 0, rows are staged with 4-element vector loads
     int bulk;                              // 1: planes are fetched one unit ahead with cp.async.bulk into raw_off
@@ -116,7 +117,7 @@ struct Geom {
     int npatch;                            // staging work items per plane (vec: 2x4 pixel patches, else 2x2 blocks)
     FastDiv d_npatch, d_prow;              // / npatch, / (patches per patch-row)
     FastDiv d_lvl[MAXL + 1], d_lvlw[MAXL + 1];  // / (Hl*Wl), / Wl   (levels >= 2 staging)
-    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase, d_bg;
+    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase, d_B;
     // weight-gradient kernel: class-major thread allocation and partial-sum slots
     int thr_start[4 * MAXL + 2];
     int np;
@@ -131,24 +132,29 @@ __host__ __device__ inline int block_of_unit(long long v, int nb, int units) {
 }
 
 // ------------------------------------------------------------------ shared device pieces
-__device__ __forceinline__ void build_weight_table(float *wtab, const Geom &g, int c, bool flip,
+__device__ __forceinline__ void build_weight_table(float *wtab, const Geom &g, int c0, bool flip,
                                                    const float *__restrict__ w0, const float *__restrict__ s0,
                                                    const float *__restrict__ b0, const float *__restrict__ wl,
                                                    const float *__restrict__ sl) {
+    // one table per plane slot (channel c0 + slot): [slot][class][WT_STRIDE], folded bias at [slot][0][25]
     const int ncls = 1 + 4 * g.L;
-    for (int e = threadIdx.x; e < ncls * KK; e += blockDim.x) {
-        const int cls = e / KK, t = e - cls * KK, src = flip ? (KK - 1 - t) : t;
-        float w;
-        if (cls == 0) {
-            w = __ldg(w0 + c * KK + src) * __ldg(s0 + c);
-        } else {
-            const int l = (cls - 1) >> 2, sub = (cls - 1) & 3;
-            const size_t i = ((size_t)l * g.C + c) * 4 + sub;
-            w = __ldg(wl + i * KK + src) * __ldg(sl + i);
+    for (int e = threadIdx.x; e < g.NPL * ncls * KK; e += blockDim.x) {
+        const int sc = e / KK, t = e - sc * KK, slot = sc / ncls, cls = sc - slot * ncls;
+        const int c = c0 + slot, src = flip ? (KK - 1 - t) : t;
+        float w = 0.f;
+        if (c < g.C) {
+            if (cls == 0) {
+                w = __ldg(w0 + c * KK + src) * __ldg(s0 + c);
+            } else {
+                const int l = (cls - 1) >> 2, sub = (cls - 1) & 3;
+                const size_t i = ((size_t)l * g.C + c) * 4 + sub;
+                w = __ldg(wl + i * KK + src) * __ldg(sl + i);
+            }
         }
-        wtab[cls * WT_STRIDE + t] = w;  // Eq. 8: scale folded into the weight
+        wtab[sc * WT_STRIDE + t] = w;  // Eq. 8: scale folded into the weight
     }
-    if (threadIdx.x == 0) wtab[KK] = b0 ? __ldg(s0 + c) * __ldg(b0 + c) : 0.f;  // spare entry of class 0
+    for (int slot = threadIdx.x; slot < g.NPL; slot += blockDim.x)
+        wtab[slot * ncls * WT_STRIDE + KK] = (b0 && c0 + slot < g.C) ? __ldg(s0 + c0 + slot) * __ldg(b0 + c0 + slot) : 0.f;
 }
 
 __device__ __forceinline__ void load_weights(const float *wt, float (&w)[KK]) {
@@ -235,7 +241,7 @@ __device__ __forceinline__ PatchD decode_patch(const Geom &g, const int *off, in
 }
 template <typename T, bool RAW>
 __device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD &p0_, const T *__restrict__ gsrc,
-                                          int img_stride, int bg, int d0 = 0, int d1 = 0, int d2 = 0) {
+                                          int nvalid, int d0 = 0, int d1 = 0, int d2 = 0) {
     if (p0_.meta >= 0) return;
     PatchD p = p0_;  // d0/d1/d2 shift the x / level-1 / level-2 targets to another set of arrays (grad_out side)
     p.xi += d0;
@@ -248,8 +254,8 @@ __device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD
     for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) a[rr][cc] = 0.f;
-    if (bg * g.NPL + slot < g.B) {
-        const T *pa = gsrc + (size_t)slot * img_stride + p.so;
+    if (slot < nvalid) {
+        const T *pa = gsrc + slot * (g.H * g.W) + p.so;  // the unit's planes are contiguous
 #pragma unroll
         for (int rr = 0; rr < 4; ++rr)
             if (rr < nrows) ld4<T, RAW>(pa + rr * W, a[rr]);
@@ -288,12 +294,13 @@ struct ItemD {    // one 4 x TH conv tile
                   // base tile: -1
     int meta;     // bit 31 valid; bits 0-9 window pitch; bits 10-19 Z pitch; bits 20-23 rows to store (0..TH);
                   // bits 24-29 parameter class (0 = base, 1 + 4(l-1) + sub = level l subband sub)
+    int slot;     // plane slot of the tile
     int dg;       // float offset from this tile's x-side array to the matching grad_out-side array (backward kernel)
 };
 __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_items, int nitems, int &bslot, int &tyy,
                                              int &txx, bool &is_base) {
     ItemD d;
-    d.src = d.wt = d.dg = 0;
+    d.src = d.wt = d.dg = d.slot = 0;
     d.z = -2;
     d.meta = 0;
     if (it >= nitems) return d;
@@ -304,7 +311,7 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         decode_level_item(g, it - slot * nlv, l, sub, ty2, tx2);
         const int pitch = g.pitch[l], zp = g.zpitch[l];
         d.src = slot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * ty2 * pitch + 4 * tx2;
-        d.wt = g.wtab_off + (1 + (l - 1) * 4 + sub) * WT_STRIDE;
+        d.wt = g.wtab_off + (slot * (1 + 4 * g.L) + 1 + (l - 1) * 4 + sub) * WT_STRIDE;
         int zleft = g.zrows[l] - TH * ty2;
         if (zleft > TH) zleft = TH;
         if (4 * tx2 < zp && zleft > 0) d.z = slot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * ty2 * zp + 4 * tx2;
@@ -312,6 +319,7 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         d.meta = (int)(0x80000000u | (unsigned)pitch | ((unsigned)zp << 10) | ((unsigned)zleft << 20) |
                        ((unsigned)(1 + (l - 1) * 4 + sub) << 24));
         d.dg = g.offG[l] - g.offA[l];
+        d.slot = slot;
     } else {
         const int bi = it - nlevel_items;
         bslot = fdiv(bi, g.d_nbase);
@@ -320,10 +328,11 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         txx = r - tyy * g.tx[0];
         const int pitch = g.pitch[0];
         d.src = bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
-        d.wt = g.wtab_off;
+        d.wt = g.wtab_off + bslot * (1 + 4 * g.L) * WT_STRIDE;
         d.z = -1;
         d.meta = (int)(0x80000000u | (unsigned)pitch);
         d.dg = g.offG[0] - g.offA[0];
+        d.slot = bslot;
         is_base = true;
     }
     return d;
@@ -337,16 +346,16 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
 // halo); images beyond the batch are written as zeros.
 template <typename T, bool RAW>
 __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *off, const T *__restrict__ src, int c,
-                                           int bg, int srank, int nstagers) {
+                                           int b, int srank, int nstagers) {
     const int H = g.H, W = g.W, HW = H * W;
     const int p0 = g.pitch[0];
-    const int slot_elems = RAW ? g.raw_slot_bytes / (int)sizeof(T) : 0;
-    const T *gsrc = RAW ? src : src + ((size_t)bg * g.NPL * g.C + c) * HW;  // image bg*NPL of channel c
-    const int img_stride = RAW ? slot_elems : g.C * HW;                      // next image of the unit (elements)
+    const T *gsrc = RAW ? src : src + ((size_t)b * g.C + c) * HW;  // channel c (first of the unit) of image b
+    const int img_stride = HW;                                     // the unit's planes are contiguous
+    const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
     if (g.L == 0) {
         for (int e = srank; e < g.NPL * HW; e += nstagers) {
             const int slot = fdiv(e, g.d_npatch), r = e - slot * HW, y = fdiv(r, g.d_prow), xx = r - y * W;
-            const bool valid = bg * g.NPL + slot < g.B;
+            const bool valid = slot < nvalid;
             sm[slot * g.slot_stride + off[0] + (y + 2) * p0 + xx + 2] =
                 valid ? ld1<T, RAW>(gsrc + (size_t)slot * img_stride + r) : 0.f;
         }
@@ -365,7 +374,7 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
             for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) a[rr][cc] = 0.f;
-            if (bg * g.NPL + slot < g.B) {
+            if (slot < nvalid) {
                 const T *pa = gsrc + (size_t)slot * img_stride + y * W + 4 * q;
 #pragma unroll
                 for (int rr = 0; rr < 4; ++rr)
@@ -412,7 +421,7 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
             const int y = 2 * i;
             const bool y1 = y + 1 < H;
             float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
-            if (bg * g.NPL + slot < g.B) {
+            if (slot < nvalid) {
                 const T *pa = gsrc + (size_t)slot * img_stride + y * W + 4 * q;
                 ld4<T, RAW>(pa, a0);
                 if (y1) ld4<T, RAW>(pa + W, a1);
@@ -442,7 +451,7 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
         const int y = 2 * i, xx = 2 * j;
         const bool x1 = xx + 1 < W, y1 = y + 1 < H;
         float a = 0.f, bq = 0.f, cq = 0.f, d = 0.f;
-        if (bg * g.NPL + slot < g.B) {
+        if (slot < nvalid) {
             const T *pa = gsrc + (size_t)slot * img_stride + y * W + xx;
             a = ld1<T, RAW>(pa);
             if (x1) bq = ld1<T, RAW>(pa + 1);
@@ -465,22 +474,17 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
     return 2;
 }
 
-// Issue the bulk copies of one unit's planes into the raw buffer (one thread): plane slot s receives image
-// bg*NPL+s of channel c; slots beyond the batch are skipped.  `extra_bytes` lets a caller that copies a
-// second tensor on the same barrier announce all bytes with one expect_tx.
+// Issue the bulk copy of one unit's planes into the raw buffer (one thread); a second tensor (grad_out) goes
+// right behind the first on the same barrier.
 template <typename T>
 __device__ __forceinline__ void issue_unit_copies(unsigned long long *bar, char *raw, const Geom &g,
-                                                  const T *__restrict__ src, const T *__restrict__ src2, int c, int bg) {
-    int nvalid = g.B - bg * g.NPL;
-    if (nvalid > g.NPL) nvalid = g.NPL;
-    const unsigned per = (unsigned)g.plane_bytes;
-    mbar_expect_tx(bar, per * nvalid * (src2 ? 2u : 1u));
-    const size_t HW = (size_t)g.H * g.W;
-    for (int s2 = 0; s2 < nvalid; ++s2) {
-        const size_t po = ((size_t)(bg * g.NPL + s2) * g.C + c) * HW;
-        bulk_g2s(raw + (size_t)s2 * g.raw_slot_bytes, src + po, per, bar);
-        if (src2) bulk_g2s(raw + (size_t)(g.NPL + s2) * g.raw_slot_bytes, src2 + po, per, bar);
-    }
+                                                  const T *__restrict__ src, const T *__restrict__ src2, int c0, int b) {
+    // the unit (NPL consecutive channels of image b) is one contiguous, 16-byte aligned chunk
+    const unsigned bytes = (unsigned)g.NPL * g.plane_bytes;
+    mbar_expect_tx(bar, bytes * (src2 ? 2u : 1u));
+    const size_t po = ((size_t)b * g.C + c0) * g.H * g.W;
+    bulk_g2s(raw, src + po, bytes, bar);
+    if (src2) bulk_g2s(raw + bytes, src2 + po, bytes, bar);
 }
 
 // Level l >= 2 from the raw LL band of level l-1 (already in shared memory).  Reads one element past
@@ -682,15 +686,16 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     if (g.bulk && tid == 0) {
         mbar_init(bar, 1);
         fence_async_smem();
-        const int c0 = u_begin / g.bgroups;
-        issue_unit_copies<T>(bar, raw, g, x, nullptr, c0, u_begin - c0 * g.bgroups);
+        const int cg0 = u_begin / g.B;
+        issue_unit_copies<T>(bar, raw, g, x, nullptr, cg0 * g.NPL, u_begin - cg0 * g.B);
     }
     __syncthreads();
     WT_TICK_INIT
     for (int u = u_begin; u < u_end; ++u) {
-        const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
+        const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
+        const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
         WT_TICK(0);
-        if (c != c_prev) {  // units are channel-major: the table survives all images of a channel
+        if (c != c_prev) {  // units are group-major: the tables survive all images of a channel group
             build_weight_table(wtab, g, c, FLIP, w0, s0, FLIP ? nullptr : b0, wl, sl);
             c_prev = c;
         }
@@ -703,26 +708,26 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             parity ^= 1u;
             WT_TICK(8);
             if (hoist_patch) {
-                run_patch<T, true>(sm, g, patch0, reinterpret_cast<const T *>(raw), g.raw_slot_bytes / (int)sizeof(T), bg);
-                run_patch<T, true>(sm, g, patch1, reinterpret_cast<const T *>(raw), g.raw_slot_bytes / (int)sizeof(T), bg);
+                run_patch<T, true>(sm, g, patch0, reinterpret_cast<const T *>(raw), nvalid);
+                run_patch<T, true>(sm, g, patch1, reinterpret_cast<const T *>(raw), nvalid);
                 lnext = 3;
             } else {
-                lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, bg, srank, nstagers);
+                lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, b, srank, nstagers);
             }
         } else if (hoist_patch) {
-            const T *gsrc = x + ((size_t)bg * g.NPL * g.C + c) * HW;
-            run_patch<T, false>(sm, g, patch0, gsrc, g.C * (int)HW, bg);
-            run_patch<T, false>(sm, g, patch1, gsrc, g.C * (int)HW, bg);
+            const T *gsrc = x + ((size_t)b * g.C + c) * HW;
+            run_patch<T, false>(sm, g, patch0, gsrc, nvalid);
+            run_patch<T, false>(sm, g, patch1, gsrc, nvalid);
             lnext = 3;
         } else {
-            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, srank, nstagers);
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, srank, nstagers);
         }
         WT_TICK(2);
         __syncthreads();
         if (g.bulk && tid == 0 && u + 1 < u_end) {  // the raw buffer is free again: fetch the next unit behind the math
             fence_async_smem();
-            const int cn = (u + 1) / g.bgroups;
-            issue_unit_copies<T>(bar, raw, g, x, nullptr, cn, (u + 1) - cn * g.bgroups);
+            const int cgn = (u + 1) / g.B;
+            issue_unit_copies<T>(bar, raw, g, x, nullptr, cgn * g.NPL, (u + 1) - cgn * g.B);
         }
         WT_TICK(3);
         for (int l = lnext; l <= L; ++l) {
@@ -767,7 +772,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 }
             }
         }
-        const float bias = wtab[KK];
+        const float bias = wtab[bslot * (1 + 4 * L) * WT_STRIDE + KK];
         WT_TICK(5);
         __syncthreads();
         WT_TICK(6);
@@ -777,9 +782,8 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #ifndef WT_ABL_NOSYNTH
             for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, bias, &acc[4 * hb]);
 #endif
-            const int b = bg * g.NPL + bslot;
-            if (b < g.B) {
-                T *oa = out + ((size_t)b * g.C + c) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
+            if (bslot < nvalid) {
+                T *oa = out + ((size_t)b * g.C + c + bslot) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
                 const bool vec = g.vec && (4 * txx + 3 < g.W);
 #pragma unroll
                 for (int r = 0; r < TH; ++r)
@@ -826,29 +830,29 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     if (g.bulk && tid == 0) {
         mbar_init(bar, 1);
         fence_async_smem();
-        const int c0 = u_begin / g.bgroups;
-        issue_unit_copies<T>(bar, raw, g, x, go, c0, u_begin - c0 * g.bgroups);
+        const int cg0 = u_begin / g.B;
+        issue_unit_copies<T>(bar, raw, g, x, go, cg0 * g.NPL, u_begin - cg0 * g.B);
     }
     __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
-        const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
+        const int c = fdiv(u, g.d_B), b = u - c * g.B;  // this kernel is planned with one plane per unit: group = channel
         int lnext;
         if (g.bulk) {
             if (!mbar_wait(bar, parity)) atomicExch(status, 1);
             parity ^= 1u;
             const T *rx = reinterpret_cast<const T *>(raw);
-            const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.raw_slot_bytes);
-            lnext = stage_input<T, true>(sm, g, g.offA, rx, c, bg, tid, nthr);
-            stage_input<T, true>(sm, g, g.offG, rg, c, bg, tid, nthr);
+            const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.plane_bytes);
+            lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, tid, nthr);
+            stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
         } else {
-            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, tid, nthr);
-            stage_input<T, false>(sm, g, g.offG, go, c, bg, tid, nthr);
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, tid, nthr);
+            stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
         }
         __syncthreads();
         if (g.bulk && tid == 0 && u + 1 < u_end) {
             fence_async_smem();
-            const int cn = (u + 1) / g.bgroups;
-            issue_unit_copies<T>(bar, raw, g, x, go, cn, (u + 1) - cn * g.bgroups);
+            const int cgn = (u + 1) / g.B;
+            issue_unit_copies<T>(bar, raw, g, x, go, cgn * g.NPL, (u + 1) - cgn * g.B);
         }
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
@@ -895,7 +899,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             }
         }
         __syncthreads();
-        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_bg) != c);
+        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_B) != c);
         if (last_of_channel) {
             // block tree through shared memory: every thread parks its 26 sums in the (now idle) array
             // region, then one thread per (class, tap) adds its class's threads in index order
@@ -904,7 +908,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             for (int t = 0; t < KK; ++t) scr[(size_t)tid * (KK + 1) + t] = acc[t];
             scr[(size_t)tid * (KK + 1) + KK] = gsum;
             __syncthreads();
-            const int slotp = blockIdx.x - block_of_unit((long long)c * g.bgroups, gridDim.x, g.units);
+            const int slotp = blockIdx.x - block_of_unit((long long)c * g.B, gridDim.x, g.units);
             for (int e = tid; e < ncls * (KK + 1); e += nthr) {
                 const int c2 = e / (KK + 1), t = e - c2 * (KK + 1);
                 if (c2 > 0 && t == KK) continue;
@@ -966,22 +970,23 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     int c_prev = -1;
     __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
-        const int c = fdiv(u, g.d_bg), bg = u - c * g.bgroups;
+        const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
+        const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
         if (c != c_prev) {
             build_weight_table(wtab, g, c, true, w0, s0, nullptr, wl, sl);
             c_prev = c;
         }
         int lnext;
         if (hoist_patch) {
-            const size_t po = ((size_t)bg * g.NPL * g.C + c) * HW;
-            run_patch<T, false>(sm, g, patch0, x + po, g.C * (int)HW, bg);
-            run_patch<T, false>(sm, g, patch0, go + po, g.C * (int)HW, bg, dA0, dA1, dA2);
-            run_patch<T, false>(sm, g, patch1, x + po, g.C * (int)HW, bg);
-            run_patch<T, false>(sm, g, patch1, go + po, g.C * (int)HW, bg, dA0, dA1, dA2);
+            const size_t po = ((size_t)b * g.C + c) * HW;
+            run_patch<T, false>(sm, g, patch0, x + po, nvalid);
+            run_patch<T, false>(sm, g, patch0, go + po, nvalid, dA0, dA1, dA2);
+            run_patch<T, false>(sm, g, patch1, x + po, nvalid);
+            run_patch<T, false>(sm, g, patch1, go + po, nvalid, dA0, dA1, dA2);
             lnext = 3;
         } else {
-            lnext = stage_input<T, false>(sm, g, g.offA, x, c, bg, tid, nthr);
-            stage_input<T, false>(sm, g, g.offG, go, c, bg, tid, nthr);
+            lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, tid, nthr);
+            stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
         }
         __syncthreads();
         for (int l = lnext; l <= L; ++l) {
@@ -1043,16 +1048,15 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             const float *S = sm + bslot * g.slot_stride;
 #pragma unroll
             for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, 0.f, &acc[4 * hb]);
-            const int b = bg * g.NPL + bslot;
-            if (b < g.B) {
-                T *oa = gx + ((size_t)b * g.C + c) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
+            if (bslot < nvalid) {
+                T *oa = gx + ((size_t)b * g.C + c + bslot) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
                 const bool vec = g.vec && (4 * txx + 3 < g.W);
 #pragma unroll
                 for (int r = 0; r < TH; ++r)
                     if (TH * tyy + r < g.H) store_row4(oa + (size_t)r * g.W, 4 * txx, g.W, vec, acc[r]);
             }
         }
-        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_bg) != c);
+        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_B) != cg);
         if (last_of_channel) {
             // block tree through shared memory: park the 26 sums and the class of every thread in the array
             // region (idle now), then one thread per (class, tap) adds its class's threads in index order
@@ -1061,20 +1065,21 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
             for (int t = 0; t < KK; ++t) scr[tid * (KK + 2) + t] = accw[t];
             scr[tid * (KK + 2) + KK] = gsum;
-            scr[tid * (KK + 2) + KK + 1] = __int_as_float(item.meta < 0 ? cls : -1);
+            scr[tid * (KK + 2) + KK + 1] = __int_as_float(item.meta < 0 ? item.slot * 64 + cls : -1);
             __syncthreads();
-            const int slotp = blockIdx.x - block_of_unit((long long)c * g.bgroups, gridDim.x, g.units);
-            for (int e = tid; e < ncls * (KK + 1); e += nthr) {
-                const int c2 = e / (KK + 1), t = e - c2 * (KK + 1);
+            const int slotp = blockIdx.x - block_of_unit((long long)cg * g.B, gridDim.x, g.units);
+            for (int e = tid; e < nvalid * ncls * (KK + 1); e += nthr) {
+                const int sc = e / (KK + 1), t = e - sc * (KK + 1), slot = sc / ncls, c2 = sc - slot * ncls;
                 if (c2 > 0 && t == KK) continue;
+                const int tag = slot * 64 + c2, ch = c + slot;
                 float sacc = 0.f;
                 for (int th = 0; th < nthr; ++th)
-                    if (__float_as_int(scr[th * (KK + 2) + KK + 1]) == c2) sacc += scr[th * (KK + 2) + t];
+                    if (__float_as_int(scr[th * (KK + 2) + KK + 1]) == tag) sacc += scr[th * (KK + 2) + t];
                 if (c2 == 0) {
-                    part0[((size_t)c * g.np + slotp) * (KK + 1) + t] = sacc;
+                    part0[((size_t)ch * g.np + slotp) * (KK + 1) + t] = sacc;
                 } else {
                     const int l = (c2 - 1) >> 2, sb_ = (c2 - 1) & 3;
-                    partl[(size_t)l * g.C * g.np * 4 * KK + (((size_t)c * g.np + slotp) * 4 + sb_) * KK + t] = sacc;
+                    partl[(size_t)l * g.C * g.np * 4 * KK + (((size_t)ch * g.np + slotp) * 4 + sb_) * KK + t] = sacc;
                 }
             }
             __syncthreads();
@@ -1122,9 +1127,8 @@ inline void fill_common(Geom &g, int B, int C, int H, int W, int L, int elem_byt
     g.d_nbase = make_fastdiv(g.nbase);
     g.npatch4 = ((H + 3) / 4) * (W / 4 > 0 ? W / 4 : 1);
     g.d_npatch4 = make_fastdiv(g.npatch4);
-    // bulk prefetch needs 16-byte aligned plane starts and sizes
     g.plane_bytes = H * W * elem_bytes;
-    g.bulk = (g.plane_bytes % 16 == 0) ? 1 : 0;
+    g.bulk = 0;  // decided per plan: a unit of NPL planes must be a 16-byte multiple and C a multiple of NPL
     g.raw_slot_bytes = g.plane_bytes;
 }
 
@@ -1134,7 +1138,7 @@ inline long long finish_layout(Geom &g, long long arrays_floats, int wtab_floats
     g.wtab_off = (int)off;
     off += pad4(wtab_floats);
     g.raw_off = (int)off;
-    if (use_bulk) off += (long long)raw_tensors * g.NPL * g.raw_slot_bytes / 4;
+    if (use_bulk) off += ((long long)raw_tensors * g.NPL * g.plane_bytes + 3) / 4;
     off = pad4((int)off);
     g.bar_off = (int)off;
     return off + 4;
@@ -1170,13 +1174,14 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
     fill_common(g, B, C, H, W, L, elem_bytes);
     const int slot = layout_slot(g, false, true);
     const int M = g.lvl_start[L + 1] + g.nbase;
-    const int wtab = (1 + 4 * L) * WT_STRIDE;
     bool found = false;
     best.score = -1.0;
     for (int npl = 1; npl <= 64; ++npl) {
-        if (npl > 1 && npl > B) break;
+        if (npl > 1 && npl > C) break;
         if (fNpl && npl != fNpl) continue;
-        for (int use_bulk = (g.bulk && !no_bulk) ? 1 : 0; use_bulk >= 0; --use_bulk) {
+        const int wtab = npl * (1 + 4 * L) * WT_STRIDE;
+        const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !no_bulk;
+        for (int use_bulk = can_bulk ? 1 : 0; use_bulk >= 0; --use_bulk) {
         Geom cg = g;
         cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
         const long long smem_floats = finish_layout(cg, (long long)npl * slot, wtab, 1, use_bulk);
@@ -1191,7 +1196,7 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
                 if (bps * (bytes + 1024) > SMEM_PER_SM) continue;
                 const int rounds = (npl * M + T - 1) / T;
                 const double eff = (double)npl * M / ((double)T * rounds);
-                const int bgroups = (B + npl - 1) / npl, units = C * bgroups;
+                const int ngroups = (C + npl - 1) / npl, units = ngroups * B;
                 int nblocks = NUM_SMS * bps;
                 if (nblocks > units) nblocks = units;
                 // thread-slot use x resident warps (about 16 hide the latency-bound phases) x phase overlap
@@ -1199,12 +1204,12 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
                 if (occ > 1.0) occ = 1.0;
                 const double overlap = bps >= 4 ? 1.0 : (bps == 3 ? 0.95 : (bps == 2 ? 0.8 : 0.55));
                 const double sc = eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) * (rounds <= 2 ? 1.0 : 0.9) *
-                                  partition_eff(units, nblocks) * ((double)B / ((double)bgroups * npl)) *
+                                  partition_eff(units, nblocks) * ((double)C / ((double)ngroups * npl)) *
                                   (1.0 - 1e-4 * T / 32.0);
                 if (sc > best.score + 1e-9) {
                     best = cg;
-                    best.smem_floats = (int)smem_floats; best.bgroups = bgroups; best.units = units;
-                    best.d_bg = make_fastdiv(bgroups);
+                    best.smem_floats = (int)smem_floats; best.ngroups = ngroups; best.units = units;
+                    best.d_B = make_fastdiv(B);
                     best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                     found = true;
                 }
@@ -1226,9 +1231,8 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
     const int ncls = 1 + 4 * L;
     bool found = false;
     best.score = -1.0;
-    for (int npl = 1; npl <= 64; ++npl) {
-        if (npl > 1 && npl > B) break;
-        if (fNpl && npl != fNpl) continue;
+    for (int npl = 1; npl <= 1; ++npl) {  // one plane per unit: a thread's class must map to one channel
+        (void)fNpl;
         for (int rounds = 1; rounds <= 64; ++rounds) {
             int thr[4 * MAXL + 2];
             int tot = 0, work = 0;
@@ -1246,7 +1250,8 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
             const long long scratch = (long long)T * (KK + 1);
             if (scratch > arrays) arrays = scratch;
             bool any = false;
-            for (int use_bulk = (g.bulk && !no_bulk) ? 1 : 0; use_bulk >= 0; --use_bulk) {
+            const bool can_bulk = (g.plane_bytes % 16 == 0) && !no_bulk;
+            for (int use_bulk = can_bulk ? 1 : 0; use_bulk >= 0; --use_bulk) {
                 Geom cg = g;
                 cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
                 const long long smem_floats = finish_layout(cg, arrays, 0, 2, use_bulk);
@@ -1257,25 +1262,24 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
                     if (bps * T > 512) continue;  // 128 registers per thread
                     if (fBps && bps != fBps) continue;
                     if (bps * (bytes + 1024) > SMEM_PER_SM) continue;
-                    const int bgroups = (B + npl - 1) / npl, units = C * bgroups;
+                    const int units = C * B;
                     int nblocks = NUM_SMS * bps;
                     if (nblocks > units) nblocks = units;
                     double occ = (double)bps * T / 512.0;
                     if (occ > 1.0) occ = 1.0;
                     const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
                     const double sc = ((double)work / ((double)T * rounds)) * (0.5 + 0.5 * occ) * overlap *
-                                      (use_bulk ? 1.0 : 0.8) * partition_eff(units, nblocks) *
-                                      ((double)B / ((double)bgroups * npl));
+                                      (use_bulk ? 1.0 : 0.8) * partition_eff(units, nblocks);
                     if (sc > best.score + 1e-9) {
                         best = cg;
                         best.smem_floats = (int)smem_floats;
-                        best.bgroups = bgroups; best.units = units; best.d_bg = make_fastdiv(bgroups);
+                        best.ngroups = C; best.units = units; best.d_B = make_fastdiv(B);
                         best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                         for (int k = 0; k <= ncls; ++k) best.thr_start[k] = thr[k];
                         int np = 1;
                         for (int ch = 0; ch < C; ++ch) {
-                            const int first = block_of_unit((long long)ch * bgroups, nblocks, units);
-                            const int last = block_of_unit((long long)(ch + 1) * bgroups - 1, nblocks, units);
+                            const int first = block_of_unit((long long)ch * B, nblocks, units);
+                            const int last = block_of_unit((long long)(ch + 1) * B - 1, nblocks, units);
                             if (last - first + 1 > np) np = last - first + 1;
                         }
                         best.np = np;
@@ -1299,13 +1303,13 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
     fill_common(g, B, C, H, W, L, elem_bytes);
     const int slot = layout_slot(g, true, true);
     const int M = g.lvl_start[L + 1] + g.nbase;
-    const int wtab = (1 + 4 * L) * WT_STRIDE;
     bool found = false;
     best.score = -1.0;
-    for (int npl = 1; npl <= 64; ++npl) {
-        if (npl > 1 && npl > B) break;
+    for (int npl = 1; npl <= 63; ++npl) {
+        if (npl > 1 && npl > C) break;
         if (fNpl && npl != fNpl) continue;
         if (npl * M > 256) break;
+        const int wtab = npl * (1 + 4 * L) * WT_STRIDE;
         const int T = (npl * M + 31) & ~31;
         Geom cg = g;
         cg.NPL = npl; cg.slot_stride = slot; cg.bulk = 0;
@@ -1319,23 +1323,23 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
             if (bps * T > 512) continue;  // 128 registers per thread
             if (fBps && bps != fBps) continue;
             if (bps * (bytes + 1024) > SMEM_PER_SM) continue;
-            const int bgroups = (B + npl - 1) / npl, units = C * bgroups;
+            const int ngroups = (C + npl - 1) / npl, units = ngroups * B;
             int nblocks = NUM_SMS * bps;
             if (nblocks > units) nblocks = units;
             double occ = (double)bps * T / 512.0;
             if (occ > 1.0) occ = 1.0;
             const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
             const double sc = ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * partition_eff(units, nblocks) *
-                              ((double)B / ((double)bgroups * npl));
+                              ((double)C / ((double)ngroups * npl));
             if (sc > best.score + 1e-9) {
                 best = cg;
                 best.smem_floats = (int)smem_floats;
-                best.bgroups = bgroups; best.units = units; best.d_bg = make_fastdiv(bgroups);
+                best.ngroups = ngroups; best.units = units; best.d_B = make_fastdiv(B);
                 best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                 int np = 1;
-                for (int ch = 0; ch < C; ++ch) {
-                    const int first = block_of_unit((long long)ch * bgroups, nblocks, units);
-                    const int last = block_of_unit((long long)(ch + 1) * bgroups - 1, nblocks, units);
+                for (int ch = 0; ch < ngroups; ++ch) {
+                    const int first = block_of_unit((long long)ch * B, nblocks, units);
+                    const int last = block_of_unit((long long)(ch + 1) * B - 1, nblocks, units);
                     if (last - first + 1 > np) np = last - first + 1;
                 }
                 best.np = np;
