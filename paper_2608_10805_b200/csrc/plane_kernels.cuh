@@ -27,7 +27,6 @@ namespace plane {
 
 constexpr int MAXL = 8;
 constexpr int KK = 25;
-constexpr int TH = 8;                        // register tile: 4 columns x TH rows
 constexpr int MAX_THREADS = 256;
 constexpr int NUM_SMS = 148;                 // planning constant (B200); plans must not depend on the device
 constexpr int SMEM_LIMIT = 227 * 1024;       // opt-in dynamic shared memory per block
@@ -99,6 +98,7 @@ struct Geom {
     int zrows[MAXL + 1], zpitch[MAXL + 1]; // conv outputs Z^l (forward kernel only)
     int offZ[MAXL + 1];
     int slot_stride;                       // floats per plane slot
+    int th;                                // register tile height: tiles are 4 columns x th rows (4 or 8)
     int NPL;                               // plane slots per work unit: NPL consecutive channels of one image (contiguous in memory)
     int tx[MAXL + 1], ty[MAXL + 1];        // 4 x TH tiles per level grid (index 0 = base)
     int lvl_start[MAXL + 2];               // per plane: first level-item of level l (1..L); [L+1] = count
@@ -310,11 +310,11 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         const int slot = fdiv(it, g.d_nlv);
         decode_level_item(g, it - slot * nlv, l, sub, ty2, tx2);
         const int pitch = g.pitch[l], zp = g.zpitch[l];
-        d.src = slot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + TH * ty2 * pitch + 4 * tx2;
+        d.src = slot * g.slot_stride + g.offA[l] + sub * g.rows[l] * pitch + g.th * ty2 * pitch + 4 * tx2;
         d.wt = g.wtab_off + (slot * (1 + 4 * g.L) + 1 + (l - 1) * 4 + sub) * WT_STRIDE;
-        int zleft = g.zrows[l] - TH * ty2;
-        if (zleft > TH) zleft = TH;
-        if (4 * tx2 < zp && zleft > 0) d.z = slot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + TH * ty2 * zp + 4 * tx2;
+        int zleft = g.zrows[l] - g.th * ty2;
+        if (zleft > g.th) zleft = g.th;
+        if (4 * tx2 < zp && zleft > 0) d.z = slot * g.slot_stride + g.offZ[l] + sub * g.zrows[l] * zp + g.th * ty2 * zp + 4 * tx2;
         if (zleft < 0) zleft = 0;
         d.meta = (int)(0x80000000u | (unsigned)pitch | ((unsigned)zp << 10) | ((unsigned)zleft << 20) |
                        ((unsigned)(1 + (l - 1) * 4 + sub) << 24));
@@ -327,7 +327,7 @@ __device__ __forceinline__ ItemD decode_item(const Geom &g, int it, int nlevel_i
         tyy = fdiv(r, g.d_tx[0]);
         txx = r - tyy * g.tx[0];
         const int pitch = g.pitch[0];
-        d.src = bslot * g.slot_stride + g.offA[0] + TH * tyy * pitch + 4 * txx;
+        d.src = bslot * g.slot_stride + g.offA[0] + g.th * tyy * pitch + 4 * txx;
         d.wt = g.wtab_off + bslot * (1 + 4 * g.L) * WT_STRIDE;
         d.z = -1;
         d.meta = (int)(0x80000000u | (unsigned)pitch);
@@ -510,6 +510,7 @@ __device__ __forceinline__ void stage_level(float *sm, const Geom &g, const int 
 // 4-column x TH-row output tile of a 5x5 correlation.  `src` = array + (TH*ty)*pitch + 4*tx is the
 // window's top-left element (the array's halo of 2 makes window row rr = output row + tap row), 16-byte
 // aligned; eight floats per window row.
+template <int TH>
 __device__ __forceinline__ void conv_tile(const float *__restrict__ src, int pitch, const float (&w)[KK],
                                           float (&acc)[TH][4]) {
 #pragma unroll
@@ -643,7 +644,7 @@ __device__ __forceinline__ void synth_block(const float *S, const Geom &g, int t
 
 // FLIP = false: out = WTConv(x).  FLIP = true: the same dataflow on grad_out with every kernel rotated
 // by 180 degrees and no bias gives grad_x.  MINB = resident blocks per SM the register budget is sized for.
-template <typename T, bool FLIP, int MAXT, int MINB>
+template <typename T, bool FLIP, int MAXT, int MINB, int TH>
 __global__ void __launch_bounds__(MAXT, MINB)
 plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0,
                  const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
@@ -744,7 +745,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 if (items[k].meta < 0) {
                     float w[KK];
                     load_weights(sm + items[k].wt, w);
-                    conv_tile(sm + items[k].src, items[k].meta & 0x3ff, w, acc);
+                    conv_tile<TH>(sm + items[k].src, items[k].meta & 0x3ff, w, acc);
                     if (items[k].z >= 0) {
                         const int zp = (items[k].meta >> 10) & 0x3ff, zleft = (items[k].meta >> 20) & 0xf;
                         float *z = sm + items[k].z;
@@ -762,7 +763,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 has_base = isb;
                 float w[KK];
                 load_weights(sm + d.wt, w);
-                conv_tile(sm + d.src, d.meta & 0x3ff, w, acc);
+                conv_tile<TH>(sm + d.src, d.meta & 0x3ff, w, acc);
                 if (d.z >= 0) {
                     const int zp = (d.meta >> 10) & 0x3ff, zleft = (d.meta >> 20) & 0xf;
                     float *z = sm + d.z;
@@ -800,7 +801,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 // dWfold^l[u,v] += sum_{i,j} D^l[i,j] Y^l[i+u-2, j+v-2] (and the base class with grad_out and x), Sec. 2.2.
 // Thread t serves class cls(t) only (class-major allocation thr_start[]); accumulators persist over all
 // units of a channel and are flushed to `part0` / `partl` when the channel changes.
-template <typename T, int MAXT, int MINB>
+template <typename T, int MAXT, int MINB, int TH>
 __global__ void __launch_bounds__(MAXT, MINB)
 plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                    float *__restrict__ part0, float *__restrict__ partl /* level l at l*C*np*100 */,
@@ -941,7 +942,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 //                    closed-form synthesis of Proposition 2 and the store of grad_x.
 // Used when a unit's item list fits one round of the block (<= 256 tiles); otherwise the separate weight-
 // gradient and input-gradient kernels run.
-template <typename T>
+template <typename T, int TH>
 __global__ void __launch_bounds__(256, 2)
 plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                  const float *__restrict__ w0, const float *__restrict__ s0, const float *__restrict__ wl,
@@ -1034,7 +1035,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             // input gradient: rotated-kernel conv of the D window
             float w[KK];
             load_weights(sm + item.wt, w);
-            conv_tile(gsrc, pitch, w, acc);
+            conv_tile<TH>(gsrc, pitch, w, acc);
             if (item.z >= 0) {
                 const int zp = (item.meta >> 10) & 0x3ff, zleft = (item.meta >> 20) & 0xf;
                 float *z = sm + item.z;
@@ -1093,8 +1094,8 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 }
 
 // ------------------------------------------------------------------ host-side planning
-inline void fill_common(Geom &g, int B, int C, int H, int W, int L, int elem_bytes) {
-    g.B = B; g.C = C; g.H = H; g.W = W; g.L = L;
+inline void fill_common(Geom &g, int B, int C, int H, int W, int L, int elem_bytes, int TH) {
+    g.B = B; g.C = C; g.H = H; g.W = W; g.L = L; g.th = TH;
     g.Hl[0] = H; g.Wl[0] = W;
     for (int l = 1; l <= MAXL; ++l) { g.Hl[l] = (g.Hl[l - 1] + 1) / 2; g.Wl[l] = (g.Wl[l - 1] + 1) / 2; }
     for (int l = 0; l <= L; ++l) {
@@ -1150,7 +1151,7 @@ inline int layout_slot(Geom &g, bool with_g, bool with_z) {
     int off = 0;
     for (int l = 0; l <= g.L; ++l) { g.offA[l] = off; off += (l == 0 ? 1 : 4) * g.rows[l] * g.pitch[l]; }
     for (int l = 0; l <= g.L; ++l) { g.offG[l] = off; if (with_g) off += (l == 0 ? 1 : 4) * g.rows[l] * g.pitch[l]; }
-    const int padH = g.ty[0] * TH, padW = g.tx[0] * 4;  // pixels the base tiles cover
+    const int padH = g.ty[0] * g.th, padW = g.tx[0] * 4;  // pixels the base tiles cover
     for (int l = 1; l <= g.L; ++l) {
         // only the coefficients the (padded) base tiles read in the synthesis are kept
         const int zr = ((padH - 1) >> l) + 1;
@@ -1166,16 +1167,26 @@ inline double partition_eff(int units, int nblocks) {
     return (double)units / ((double)per * nblocks);
 }
 
+// Useful conv outputs over tile slots issued, times a small penalty for the per-tile overhead of short tiles.
+inline double tile_score(const Geom &g) {
+    double useful = (double)g.H * g.W, slots = (double)g.nbase * 4 * g.th;
+    for (int l = 1; l <= g.L; ++l) {
+        useful += 4.0 * g.Hl[l] * g.Wl[l];
+        slots += 4.0 * g.tx[l] * g.ty[l] * 4 * g.th;
+    }
+    return useful / slots * (g.th == 8 ? 1.0 : 0.93);
+}
+
 // Forward plan.  `tune` (0 = automatic): bits 0-4 threads/32, bits 5-7 blocks per SM, bits 8-13 planes per unit.
-inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+inline bool plan_forward_th(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune, int th) {
     const int fT = (tune & 31) * 32, fBps = (tune >> 5) & 7, fNpl = (tune >> 8) & 63;
     const bool no_bulk = (tune >> 23) & 1;
     Geom g = {};
-    fill_common(g, B, C, H, W, L, elem_bytes);
+    fill_common(g, B, C, H, W, L, elem_bytes, th);
     const int slot = layout_slot(g, false, true);
     const int M = g.lvl_start[L + 1] + g.nbase;
+    const double teff = tile_score(g);
     bool found = false;
-    best.score = -1.0;
     for (int npl = 1; npl <= 64; ++npl) {
         if (npl > 1 && npl > C) break;
         if (fNpl && npl != fNpl) continue;
@@ -1203,7 +1214,7 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
                 double occ = (double)bps * T / 384.0;
                 if (occ > 1.0) occ = 1.0;
                 const double overlap = bps >= 4 ? 1.0 : (bps == 3 ? 0.95 : (bps == 2 ? 0.8 : 0.55));
-                const double sc = eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) * (rounds <= 2 ? 1.0 : 0.9) *
+                const double sc = teff * eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) * (rounds <= 2 ? 1.0 : 0.9) *
                                   partition_eff(units, nblocks) * ((double)C / ((double)ngroups * npl)) *
                                   (1.0 - 1e-4 * T / 32.0);
                 if (sc > best.score + 1e-9) {
@@ -1222,15 +1233,15 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
 
 // Weight-gradient plan: per class c with n_c tiles (x NPL) allocate ceil(n_c NPL / rounds) threads, smallest
 // `rounds` that fits the thread limit.  tune bits 14-19: planes per unit, bits 20-22: blocks per SM.
-inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+inline bool plan_wgrad_th(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune, int th) {
     const int fNpl = (tune >> 14) & 63, fBps = (tune >> 20) & 7;
     const bool no_bulk = (tune >> 23) & 1;
     Geom g = {};
-    fill_common(g, B, C, H, W, L, elem_bytes);
+    fill_common(g, B, C, H, W, L, elem_bytes, th);
     const int slot = layout_slot(g, true, false);
     const int ncls = 1 + 4 * L;
+    const double teff = tile_score(g);
     bool found = false;
-    best.score = -1.0;
     for (int npl = 1; npl <= 1; ++npl) {  // one plane per unit: a thread's class must map to one channel
         (void)fNpl;
         for (int rounds = 1; rounds <= 64; ++rounds) {
@@ -1268,7 +1279,7 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
                     double occ = (double)bps * T / 512.0;
                     if (occ > 1.0) occ = 1.0;
                     const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
-                    const double sc = ((double)work / ((double)T * rounds)) * (0.5 + 0.5 * occ) * overlap *
+                    const double sc = teff * ((double)work / ((double)T * rounds)) * (0.5 + 0.5 * occ) * overlap *
                                       (use_bulk ? 1.0 : 0.8) * partition_eff(units, nblocks);
                     if (sc > best.score + 1e-9) {
                         best = cg;
@@ -1296,15 +1307,14 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
 
 // Fused-backward plan: one round (every tile its own thread), both input pyramids plus Z in shared memory, no
 // bulk prefetch.  tune bits 14-19: planes per unit, bits 20-22: blocks per SM (shared with the weight-gradient plan).
-inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune, int th) {
     const int fNpl = (tune >> 14) & 63, fBps = (tune >> 20) & 7;
-    if ((tune >> 24) & 1) return false;  // bit 24: never fuse
     Geom g = {};
-    fill_common(g, B, C, H, W, L, elem_bytes);
+    fill_common(g, B, C, H, W, L, elem_bytes, th);
     const int slot = layout_slot(g, true, true);
     const int M = g.lvl_start[L + 1] + g.nbase;
+    const double teff = tile_score(g);
     bool found = false;
-    best.score = -1.0;
     for (int npl = 1; npl <= 63; ++npl) {
         if (npl > 1 && npl > C) break;
         if (fNpl && npl != fNpl) continue;
@@ -1329,7 +1339,7 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
             double occ = (double)bps * T / 512.0;
             if (occ > 1.0) occ = 1.0;
             const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
-            const double sc = ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * partition_eff(units, nblocks) *
+            const double sc = teff * ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * partition_eff(units, nblocks) *
                               ((double)C / ((double)ngroups * npl));
             if (sc > best.score + 1e-9) {
                 best = cg;
@@ -1348,6 +1358,30 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
         }
     }
     return found;
+}
+
+// Each plan is searched for both tile heights; tune bit 25 forces 8 rows, bit 26 forces 4 rows.
+inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    best.score = -1.0;
+    bool ok = false;
+    if (!((tune >> 26) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 8);
+    if (!((tune >> 25) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    return ok;
+}
+inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    best.score = -1.0;
+    bool ok = false;
+    if (!((tune >> 26) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 8);
+    if (!((tune >> 25) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    return ok;
+}
+inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    if ((tune >> 24) & 1) return false;  // bit 24: never fuse
+    best.score = -1.0;
+    bool ok = false;
+    if (!((tune >> 26) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 8);
+    if (!((tune >> 25) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    return ok;
 }
 
 inline int dtype_bytes(int dtype) { return dtype == 0 ? 4 : 2; }
@@ -1373,13 +1407,14 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
                        const float *sl, T *out, int *status, cudaStream_t st) {
     cudaError_t e;
     const size_t smem = (size_t)g.smem_floats * 4;
-#define WT_LAUNCH_FWD(MAXT_, MINB_)                                                                 \
+#define WT_LAUNCH_FWD_TH(MAXT_, MINB_, TH_)                                                         \
     {                                                                                               \
-        auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_>;                                        \
+        auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_, TH_>;                                   \
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);    \
         if (e != cudaSuccess) return e;                                                             \
         kern<<<g.nblocks, g.nthreads, smem, st>>>(g, x, w0, s0, b0, wl, sl, out, status);           \
     }
+#define WT_LAUNCH_FWD(MAXT_, MINB_) { if (g.th == 8) WT_LAUNCH_FWD_TH(MAXT_, MINB_, 8) else WT_LAUNCH_FWD_TH(MAXT_, MINB_, 4) }
     if (g.nthreads <= 128 && g.blocks_per_sm <= 3) {
         WT_LAUNCH_FWD(128, 3)
     } else if (g.nthreads * g.blocks_per_sm <= 512) {
@@ -1388,6 +1423,7 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
         if (g.nthreads <= 128) WT_LAUNCH_FWD(128, 6) else WT_LAUNCH_FWD(256, 3)
     }
 #undef WT_LAUNCH_FWD
+#undef WT_LAUNCH_FWD_TH
     return cudaGetLastError();
 }
 
@@ -1412,10 +1448,17 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
         cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // partial slots no block writes must read as zero
         if (e != cudaSuccess) return e;
-        auto kb = plane_bwd_kernel<T>;
-        e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-        if (e != cudaSuccess) return e;
-        kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl);
+        if (gw.th == 8) {
+            auto kb = plane_bwd_kernel<T, 8>;
+            e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+            if (e != cudaSuccess) return e;
+            kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl);
+        } else {
+            auto kb = plane_bwd_kernel<T, 4>;
+            e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+            if (e != cudaSuccess) return e;
+            kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl);
+        }
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         ep->part0 = part0;
         ep->np0 = gw.np;
@@ -1434,17 +1477,19 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
     cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // status word; partial slots no block writes must read as zero
     if (e != cudaSuccess) return e;
     const size_t smem = (size_t)gw.smem_floats * 4;
-    if (gw.nthreads <= 128) {
-        auto kw = plane_wgrad_kernel<T, 128, 4>;
-        e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-        if (e != cudaSuccess) return e;
-        kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);
-    } else {
-        auto kw = plane_wgrad_kernel<T, 256, 2>;
-        e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-        if (e != cudaSuccess) return e;
-        kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);
+#define WT_LAUNCH_WG(MAXT_, MINB_, TH_)                                                            \
+    {                                                                                              \
+        auto kw = plane_wgrad_kernel<T, MAXT_, MINB_, TH_>;                                        \
+        e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);     \
+        if (e != cudaSuccess) return e;                                                            \
+        kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);                \
     }
+    if (gw.nthreads <= 128) {
+        if (gw.th == 8) WT_LAUNCH_WG(128, 4, 8) else WT_LAUNCH_WG(128, 4, 4)
+    } else {
+        if (gw.th == 8) WT_LAUNCH_WG(256, 2, 8) else WT_LAUNCH_WG(256, 2, 4)
+    }
+#undef WT_LAUNCH_WG
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = launch_fwd<T, true>(gf, go, w0, s0, nullptr, wl, sl, gx, status, st)) != cudaSuccess) return e;
     ep->part0 = part0;
