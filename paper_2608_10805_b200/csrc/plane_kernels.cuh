@@ -64,6 +64,14 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
     }
     return false;
 }
+// shared -> global bulk store (same alignment rules); completion is tracked per thread in bulk groups
+__device__ __forceinline__ void bulk_s2g(void *gdst, const void *src, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_addr(src)), "r"(bytes)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// wait until every bulk store this thread issued has finished READING its shared-memory source
+__device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // order earlier generic-proxy accesses of shared memory before later async-proxy (bulk copy) writes
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -112,6 +120,7 @@ struct Geom {
     int bulk;                              // 1: planes are fetched one unit ahead with cp.async.bulk into raw_off
     int raw_off, raw_slot_bytes, plane_bytes;  // raw staging buffer (float offset), bytes per plane slot / per plane
     int bar_off;                           // float offset of the copy mbarrier (8-byte aligned)
+    int bulk_out, out_off;                 // 1: results are assembled in shared memory (out_off) and leave with one bulk store
     int npatch4;                           // 4x4 pixel patches per plane (vec staging of levels 1 and 2 in one pass)
     FastDiv d_npatch4;
     int npatch;                            // staging work items per plane (vec: 2x4 pixel patches, else 2x2 blocks)
@@ -582,6 +591,30 @@ __device__ __forceinline__ void store_row4(__nv_bfloat16 *__restrict__ p, int x0
     }
 }
 
+// Store one finished 4 x TH tile: straight to global memory (vector rows where the width allows), or, in
+// bulk-out mode, element by element into the unit's shared-memory image that one bulk store sends out.
+template <typename T, int TH>
+__device__ __forceinline__ void store_tile(const Geom &g, float *sm, T *__restrict__ gplane, int bslot, int tyy, int txx,
+                                           float (&acc)[TH][4]) {
+    if (g.bulk_out) {
+        T *ob = reinterpret_cast<T *>(sm + g.out_off) + bslot * (g.H * g.W) + (TH * tyy) * g.W + 4 * txx;
+#pragma unroll
+        for (int r = 0; r < TH; ++r) {
+            if (TH * tyy + r < g.H) {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    if (4 * txx + cc < g.W) stf(ob + r * g.W + cc, acc[r][cc]);
+            }
+        }
+    } else {
+        T *oa = gplane + (size_t)(TH * tyy) * g.W + 4 * txx;
+        const bool vec = g.vec && (4 * txx + 3 < g.W);
+#pragma unroll
+        for (int r = 0; r < TH; ++r)
+            if (TH * tyy + r < g.H) store_row4(oa + (size_t)r * g.W, 4 * txx, g.W, vec, acc[r]);
+    }
+}
+
 // ------------------------------------------------------------------ forward / input-gradient kernel
 // Adds the Proposition 2 terms of all levels to one 4x4 pixel block (block row t4, block column tx of
 // the plane) held in a[0..3][0..3]; `bias` is the folded bias.
@@ -669,7 +702,10 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     // down to a warp) while the others run the previous unit's synthesis; if those are too few, by everybody.
     int nstagers = (nlevel_items / 32) * 32;
     if (nstagers > nthr) nstagers = nthr;
-    if (nstagers * 4 < nthr) nstagers = nthr;
+    {   // staging work items of one unit; more than two per stager: everybody stages
+        const int nwork = g.NPL * (L == 0 ? g.H * g.W : ((g.vec && L >= 2) ? g.npatch4 : g.npatch));
+        if (nstagers * 4 < nthr || nwork > 2 * nstagers) nstagers = nthr;
+    }
     const int srank = tid < nstagers ? tid : 0x3fffffff;
     // hoisted descriptors: two tiles and two staging patches per thread cover the plans in use
     constexpr int MAXI = 2;
@@ -775,6 +811,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         }
         const float bias = wtab[bslot * (1 + 4 * L) * WT_STRIDE + KK];
         WT_TICK(5);
+        if (g.bulk_out && tid == 0) bulk_store_wait_read();  // the previous unit's store has drained the output image
         __syncthreads();
         WT_TICK(6);
         if (has_base) {
@@ -783,18 +820,20 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #ifndef WT_ABL_NOSYNTH
             for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, bias, &acc[4 * hb]);
 #endif
-            if (bslot < nvalid) {
-                T *oa = out + ((size_t)b * g.C + c + bslot) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
-                const bool vec = g.vec && (4 * txx + 3 < g.W);
-#pragma unroll
-                for (int r = 0; r < TH; ++r)
-                    if (TH * tyy + r < g.H) store_row4(oa + (size_t)r * g.W, 4 * txx, g.W, vec, acc[r]);
+            if (bslot < nvalid) store_tile<T, TH>(g, sm, out + ((size_t)b * g.C + c + bslot) * HW, bslot, tyy, txx, acc);
+        }
+        if (g.bulk_out) {  // the unit is contiguous in global memory: one bulk store once every tile is in place
+            __syncthreads();
+            if (tid == 0) {
+                fence_async_smem();
+                bulk_s2g(out + ((size_t)b * g.C + c) * HW, sm + g.out_off, (unsigned)g.NPL * g.plane_bytes);
             }
         }
         WT_TICK(7);
         // The next unit's staging overwrites x / Y (last read before the barrier above) and possibly the
         // weight table (bias already in a register); Z is next written after the staging barriers.
     }
+    if (g.bulk_out && tid == 0) bulk_store_wait_read();  // shared memory must outlive the last bulk store's reads
 }
 
 // ------------------------------------------------------------------ weight-gradient kernel
@@ -942,16 +981,19 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 //                    closed-form synthesis of Proposition 2 and the store of grad_x.
 // Used when a unit's item list fits one round of the block (<= 256 tiles); otherwise the separate weight-
 // gradient and input-gradient kernels run.
-template <typename T, int TH>
+template <typename T, int TH, bool BULK>
 __global__ void __launch_bounds__(256, 2)
 plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                  const float *__restrict__ w0, const float *__restrict__ s0, const float *__restrict__ wl,
                  const float *__restrict__ sl, T *__restrict__ gx, float *__restrict__ part0,
-                 float *__restrict__ partl /* level l at l*C*np*100 */) {
+                 float *__restrict__ partl /* level l at l*C*np*100 */, int *__restrict__ status) {
     extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
     for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
     float *wtab = sm + g.wtab_off;
+    unsigned long long *bar = reinterpret_cast<unsigned long long *>(sm + g.bar_off);
+    char *raw = reinterpret_cast<char *>(sm + g.raw_off);
+    unsigned parity = 0;
     const int L = g.L, nlv = g.lvl_start[L + 1], ncls = 1 + 4 * L;
     const int nlevel_items = g.NPL * nlv, nitems = nlevel_items + g.NPL * g.nbase;
     const size_t HW = (size_t)g.H * g.W;
@@ -970,6 +1012,13 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     for (int t = 0; t < KK; ++t) accw[t] = 0.f;
     int c_prev = -1;
     __syncthreads();
+    if (BULK && tid == 0) {
+        mbar_init(bar, 1);
+        fence_async_smem();
+        const int cg0 = u_begin / g.B;
+        issue_unit_copies<T>(bar, raw, g, x, go, cg0 * g.NPL, u_begin - cg0 * g.B);
+    }
+    __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
         const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
         const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
@@ -978,7 +1027,22 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             c_prev = c;
         }
         int lnext;
-        if (hoist_patch) {
+        if (BULK) {
+            if (!mbar_wait(bar, parity)) atomicExch(status, 1);
+            parity ^= 1u;
+            const T *rx = reinterpret_cast<const T *>(raw);
+            const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.plane_bytes);
+            if (hoist_patch) {
+                run_patch<T, true>(sm, g, patch0, rx, nvalid);
+                run_patch<T, true>(sm, g, patch0, rg, nvalid, dA0, dA1, dA2);
+                run_patch<T, true>(sm, g, patch1, rx, nvalid);
+                run_patch<T, true>(sm, g, patch1, rg, nvalid, dA0, dA1, dA2);
+                lnext = 3;
+            } else {
+                lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, tid, nthr);
+                stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
+            }
+        } else if (hoist_patch) {
             const size_t po = ((size_t)b * g.C + c) * HW;
             run_patch<T, false>(sm, g, patch0, x + po, nvalid);
             run_patch<T, false>(sm, g, patch0, go + po, nvalid, dA0, dA1, dA2);
@@ -990,6 +1054,11 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
         }
         __syncthreads();
+        if (BULK && tid == 0 && u + 1 < u_end) {
+            fence_async_smem();
+            const int cgn = (u + 1) / g.B;
+            issue_unit_copies<T>(bar, raw, g, x, go, cgn * g.NPL, (u + 1) - cgn * g.B);
+        }
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
             stage_level(sm, g, g.offG, l);
@@ -1044,17 +1113,19 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                     if (r < zleft) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
             }
         }
+        if (BULK && g.bulk_out && tid == 0) bulk_store_wait_read();  // the previous unit's store has drained the output image
         __syncthreads();
         if (has_base) {
             const float *S = sm + bslot * g.slot_stride;
 #pragma unroll
             for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, 0.f, &acc[4 * hb]);
-            if (bslot < nvalid) {
-                T *oa = gx + ((size_t)b * g.C + c + bslot) * HW + (size_t)(TH * tyy) * g.W + 4 * txx;
-                const bool vec = g.vec && (4 * txx + 3 < g.W);
-#pragma unroll
-                for (int r = 0; r < TH; ++r)
-                    if (TH * tyy + r < g.H) store_row4(oa + (size_t)r * g.W, 4 * txx, g.W, vec, acc[r]);
+            if (bslot < nvalid) store_tile<T, TH>(g, sm, gx + ((size_t)b * g.C + c + bslot) * HW, bslot, tyy, txx, acc);
+        }
+        if (BULK && g.bulk_out) {
+            __syncthreads();
+            if (tid == 0) {
+                fence_async_smem();
+                bulk_s2g(gx + ((size_t)b * g.C + c) * HW, sm + g.out_off, (unsigned)g.NPL * g.plane_bytes);
             }
         }
         const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_B) != cg);
@@ -1091,6 +1162,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         }
         __syncthreads();  // arrays and Z are free again for the next unit's staging
     }
+    if (BULK && g.bulk_out && tid == 0) bulk_store_wait_read();
 }
 
 // ------------------------------------------------------------------ host-side planning
@@ -1140,6 +1212,10 @@ inline long long finish_layout(Geom &g, long long arrays_floats, int wtab_floats
     off += pad4(wtab_floats);
     g.raw_off = (int)off;
     if (use_bulk) off += ((long long)raw_tensors * g.NPL * g.plane_bytes + 3) / 4;
+    off = pad4((int)off);
+    g.out_off = (int)off;
+    g.bulk_out = (use_bulk && !g.vec) ? 1 : 0;  // rows that are not 16-byte multiples: assemble the unit on chip
+    if (g.bulk_out) off += ((long long)g.NPL * g.plane_bytes + 3) / 4;
     off = pad4((int)off);
     g.bar_off = (int)off;
     return off + 4;
@@ -1321,14 +1397,18 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
         if (npl * M > 256) break;
         const int wtab = npl * (1 + 4 * L) * WT_STRIDE;
         const int T = (npl * M + 31) & ~31;
-        Geom cg = g;
-        cg.NPL = npl; cg.slot_stride = slot; cg.bulk = 0;
         long long arrays = (long long)npl * slot;
         const long long scratch = (long long)T * (KK + 2);
         if (scratch > arrays) arrays = scratch;
-        const long long smem_floats = finish_layout(cg, arrays, wtab, 0, false);
+        const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 23) & 1);
+        bool any = false;
+        for (int use_bulk = can_bulk ? 1 : 0; use_bulk >= 0; --use_bulk) {
+        Geom cg = g;
+        cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
+        const long long smem_floats = finish_layout(cg, arrays, wtab, 2, use_bulk);
         const long long bytes = smem_floats * 4;
-        if (bytes > SMEM_LIMIT) break;
+        if (bytes > SMEM_LIMIT) continue;
+        any = true;
         for (int bps = 1; bps <= 4; ++bps) {
             if (bps * T > 512) continue;  // 128 registers per thread
             if (fBps && bps != fBps) continue;
@@ -1339,8 +1419,8 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
             double occ = (double)bps * T / 512.0;
             if (occ > 1.0) occ = 1.0;
             const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
-            const double sc = teff * ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * partition_eff(units, nblocks) *
-                              ((double)C / ((double)ngroups * npl));
+            const double sc = teff * ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.85) *
+                              partition_eff(units, nblocks) * ((double)C / ((double)ngroups * npl));
             if (sc > best.score + 1e-9) {
                 best = cg;
                 best.smem_floats = (int)smem_floats;
@@ -1356,6 +1436,8 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
                 found = true;
             }
         }
+        }
+        if (!any) break;
     }
     return found;
 }
@@ -1448,17 +1530,20 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
         cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // partial slots no block writes must read as zero
         if (e != cudaSuccess) return e;
+#define WT_LAUNCH_BWD(TH_, BULK_)                                                                          \
+    {                                                                                                      \
+        auto kb = plane_bwd_kernel<T, TH_, BULK_>;                                                         \
+        e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);             \
+        if (e != cudaSuccess) return e;                                                                    \
+        kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl, \
+                                                                         reinterpret_cast<int *>(ws));     \
+    }
         if (gw.th == 8) {
-            auto kb = plane_bwd_kernel<T, 8>;
-            e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-            if (e != cudaSuccess) return e;
-            kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl);
+            if (gw.bulk) WT_LAUNCH_BWD(8, true) else WT_LAUNCH_BWD(8, false)
         } else {
-            auto kb = plane_bwd_kernel<T, 4>;
-            e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
-            if (e != cudaSuccess) return e;
-            kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl);
+            if (gw.bulk) WT_LAUNCH_BWD(4, true) else WT_LAUNCH_BWD(4, false)
         }
+#undef WT_LAUNCH_BWD
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         ep->part0 = part0;
         ep->np0 = gw.np;
