@@ -76,12 +76,17 @@ typedef enum {
  *   bits  8-12  threads per block / 32 of the forward / input-gradient kernel
  *   bits 13-15  resident blocks per SM of that kernel
  *   bits 16-21  planes per work unit of that kernel
- *   bits 22-27  planes per work unit of the weight-gradient kernel
- *   bits 28-30  resident blocks per SM of the weight-gradient kernel
+ *   bits 22-27  planes per work unit of the backward kernels
+ *   bit  28     never prefetch with bulk copies      bit 29  never use the fused backward kernel
+ *   bit  30     only 4 x 8 register tiles            bit 31  only 4 x 4 register tiles
  * An override that cannot be met (shared memory, registers) makes the call fail with WTCONV_ERR_CUDA. */
-#define WTCONV_TUNE(threads, blocks_per_sm, planes, wgrad_planes, wgrad_blocks_per_sm)                    \
+#define WTCONV_TUNE(threads, blocks_per_sm, planes, bwd_planes)                                            \
     ((((uint32_t)(threads) / 32u) << 8) | ((uint32_t)(blocks_per_sm) << 13) | ((uint32_t)(planes) << 16) | \
-     ((uint32_t)(wgrad_planes) << 22) | ((uint32_t)(wgrad_blocks_per_sm) << 28))
+     ((uint32_t)(bwd_planes) << 22))
+#define WTCONV_TUNE_NO_BULK (1u << 28)
+#define WTCONV_TUNE_NO_FUSED_BWD (1u << 29)
+#define WTCONV_TUNE_TILE_8 (1u << 30)
+#define WTCONV_TUNE_TILE_4 (1u << 31)
 
 typedef struct {
     int32_t B, C, H, W; /* activation shape */

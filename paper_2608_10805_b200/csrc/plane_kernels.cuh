@@ -775,37 +775,32 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         // ---- one item list: level tiles (Z^l = Wfold^l (*) Y^l) first, base tiles last; a thread's last
         //      item may be a base tile, which stays in registers across the barrier
         float acc[TH][4];
-        if (hoist_items) {
-#pragma unroll
-            for (int k = 0; k < MAXI; ++k) {
-                if (items[k].meta < 0) {
+        {
+            // one copy of the (large, fully unrolled) tile code serves every item: the loop is kept rolled and
+            // the descriptor is either one of the two hoisted ones or decoded on the spot
+            const int nmine = hoist_items ? MAXI : (nitems - tid + nthr - 1) / nthr;
+            if (!hoist_items) has_base = false;
+#pragma unroll 1
+            for (int k = 0; k < nmine; ++k) {
+                ItemD d;
+                if (hoist_items) {
+                    d = k == 0 ? items[0] : items[1];
+                } else {
+                    bool isb = false;
+                    d = decode_item(g, tid + k * nthr, nlevel_items, nitems, bslot, tyy, txx, isb);
+                    has_base = isb;
+                }
+                if (d.meta < 0) {
                     float w[KK];
-                    load_weights(sm + items[k].wt, w);
-                    conv_tile<TH>(sm + items[k].src, items[k].meta & 0x3ff, w, acc);
-                    if (items[k].z >= 0) {
-                        const int zp = (items[k].meta >> 10) & 0x3ff, zleft = (items[k].meta >> 20) & 0xf;
-                        float *z = sm + items[k].z;
+                    load_weights(sm + d.wt, w);
+                    conv_tile<TH>(sm + d.src, d.meta & 0x3ff, w, acc);
+                    if (d.z >= 0) {
+                        const int zp = (d.meta >> 10) & 0x3ff, zleft = (d.meta >> 20) & 0xf;
+                        float *z = sm + d.z;
 #pragma unroll
                         for (int r = 0; r < TH; ++r)
                             if (r < zleft) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
                     }
-                }
-            }
-        } else {
-            has_base = false;
-            for (int it = tid; it < nitems; it += nthr) {
-                bool isb = false;
-                const ItemD d = decode_item(g, it, nlevel_items, nitems, bslot, tyy, txx, isb);
-                has_base = isb;
-                float w[KK];
-                load_weights(sm + d.wt, w);
-                conv_tile<TH>(sm + d.src, d.meta & 0x3ff, w, acc);
-                if (d.z >= 0) {
-                    const int zp = (d.meta >> 10) & 0x3ff, zleft = (d.meta >> 20) & 0xf;
-                    float *z = sm + d.z;
-#pragma unroll
-                    for (int r = 0; r < TH; ++r)
-                        if (r < zleft) *reinterpret_cast<float4 *>(z + r * zp) = make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
                 }
             }
         }
@@ -1256,7 +1251,7 @@ inline double tile_score(const Geom &g) {
 // Forward plan.  `tune` (0 = automatic): bits 0-4 threads/32, bits 5-7 blocks per SM, bits 8-13 planes per unit.
 inline bool plan_forward_th(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune, int th) {
     const int fT = (tune & 31) * 32, fBps = (tune >> 5) & 7, fNpl = (tune >> 8) & 63;
-    const bool no_bulk = (tune >> 23) & 1;
+    const bool no_bulk = (tune >> 20) & 1;
     Geom g = {};
     fill_common(g, B, C, H, W, L, elem_bytes, th);
     const int slot = layout_slot(g, false, true);
@@ -1308,10 +1303,10 @@ inline bool plan_forward_th(int B, int C, int H, int W, int L, int elem_bytes, G
 }
 
 // Weight-gradient plan: per class c with n_c tiles (x NPL) allocate ceil(n_c NPL / rounds) threads, smallest
-// `rounds` that fits the thread limit.  tune bits 14-19: planes per unit, bits 20-22: blocks per SM.
+// `rounds` that fits the thread limit.  tune bits 14-19: planes per unit.
 inline bool plan_wgrad_th(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune, int th) {
-    const int fNpl = (tune >> 14) & 63, fBps = (tune >> 20) & 7;
-    const bool no_bulk = (tune >> 23) & 1;
+    const int fNpl = (tune >> 14) & 63, fBps = 0;
+    const bool no_bulk = (tune >> 20) & 1;
     Geom g = {};
     fill_common(g, B, C, H, W, L, elem_bytes, th);
     const int slot = layout_slot(g, true, false);
@@ -1382,9 +1377,9 @@ inline bool plan_wgrad_th(int B, int C, int H, int W, int L, int elem_bytes, Geo
 }
 
 // Fused-backward plan: one round (every tile its own thread), both input pyramids plus Z in shared memory, no
-// bulk prefetch.  tune bits 14-19: planes per unit, bits 20-22: blocks per SM (shared with the weight-gradient plan).
+// bulk prefetch unless it fits.  tune bits 14-19: planes per unit (shared with the weight-gradient plan).
 inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune, int th) {
-    const int fNpl = (tune >> 14) & 63, fBps = (tune >> 20) & 7;
+    const int fNpl = (tune >> 14) & 63, fBps = 0;
     Geom g = {};
     fill_common(g, B, C, H, W, L, elem_bytes, th);
     const int slot = layout_slot(g, true, true);
@@ -1400,7 +1395,7 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
         long long arrays = (long long)npl * slot;
         const long long scratch = (long long)T * (KK + 2);
         if (scratch > arrays) arrays = scratch;
-        const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 23) & 1);
+        const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 20) & 1);
         bool any = false;
         for (int use_bulk = can_bulk ? 1 : 0; use_bulk >= 0; --use_bulk) {
         Geom cg = g;
@@ -1442,27 +1437,27 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
     return found;
 }
 
-// Each plan is searched for both tile heights; tune bit 25 forces 8 rows, bit 26 forces 4 rows.
+// Each plan is searched for both tile heights; tune bit 22 forces 8 rows, bit 23 forces 4 rows.
 inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
     best.score = -1.0;
     bool ok = false;
-    if (!((tune >> 26) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 8);
-    if (!((tune >> 25) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    if (!((tune >> 23) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 8);
+    if (!((tune >> 22) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 4);
     return ok;
 }
 inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
     best.score = -1.0;
     bool ok = false;
-    if (!((tune >> 26) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 8);
-    if (!((tune >> 25) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    if (!((tune >> 23) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 8);
+    if (!((tune >> 22) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 4);
     return ok;
 }
 inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
-    if ((tune >> 24) & 1) return false;  // bit 24: never fuse
+    if ((tune >> 21) & 1) return false;  // bit 21: never fuse
     best.score = -1.0;
     bool ok = false;
-    if (!((tune >> 26) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 8);
-    if (!((tune >> 25) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    if (!((tune >> 23) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 8);
+    if (!((tune >> 22) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 4);
     return ok;
 }
 
