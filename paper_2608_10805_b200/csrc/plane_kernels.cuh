@@ -526,11 +526,16 @@ __device__ __forceinline__ void conv_tile(const float *__restrict__ src, int pit
     for (int r = 0; r < TH; ++r)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
+    // the next window row is fetched while the current one is being used (software pipelining by hand)
+    float4 n0 = *reinterpret_cast<const float4 *>(src);
+    float4 n1 = *reinterpret_cast<const float4 *>(src + 4);
 #pragma unroll
     for (int rr = 0; rr < TH + 4; ++rr) {
-        const float4 q0 = *reinterpret_cast<const float4 *>(src + rr * pitch);
-        const float4 q1 = *reinterpret_cast<const float4 *>(src + rr * pitch + 4);
-        const float in[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+        const float in[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+        if (rr + 1 < TH + 4) {
+            n0 = *reinterpret_cast<const float4 *>(src + (rr + 1) * pitch);
+            n1 = *reinterpret_cast<const float4 *>(src + (rr + 1) * pitch + 4);
+        }
 #pragma unroll
         for (int u = 0; u < 5; ++u) {
             const int r = rr - u;
