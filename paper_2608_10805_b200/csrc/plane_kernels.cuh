@@ -32,6 +32,7 @@ constexpr int NUM_SMS = 148;                 // planning constant (B200); plans 
 constexpr int SMEM_LIMIT = 227 * 1024;       // opt-in dynamic shared memory per block
 constexpr int SMEM_PER_SM = 228 * 1024;      // per SM, 1 KB reserved per resident block
 constexpr int WT_STRIDE = 28;                // floats per class in the weight table (25 taps, 16-byte padded)
+constexpr int MAX_STAGES = 4;               // deepest prefetch ring (units in flight per block)
 constexpr unsigned WAIT_LIMIT = 1u << 20;    // bounded number of (suspending) waits on the copy barrier: never an endless loop
 
 // ------------------------------------------------------------------ bulk-copy (TMA, untiled) helpers
@@ -117,9 +118,10 @@ struct Geom {
                                            // weights and gradient accumulators while it walks through the images)
     int nthreads, nblocks, blocks_per_sm;
     int vec;                               // 1: W % 4 == 0, rows are staged with 4-element vector loads
-    int bulk;                              // 1: planes are fetched one unit ahead with cp.async.bulk into raw_off
+    int bulk;                              // 1: planes are fetched ahead with cp.async.bulk into a ring of raw buffers at raw_off
+    int nstage, stage_bytes;               // ring depth (units in flight) and bytes per ring entry
     int raw_off, raw_slot_bytes, plane_bytes;  // raw staging buffer (float offset), bytes per plane slot / per plane
-    int bar_off;                           // float offset of the copy mbarrier (8-byte aligned)
+    int bar_off;                           // float offset of the ring's mbarriers (8-byte aligned, one per entry)
     int bulk_out, out_off;                 // 1: results are assembled in shared memory (out_off) and leave with one bulk store
     int npatch4;                           // 4x4 pixel patches per plane (vec staging of levels 1 and 2 in one pass)
     FastDiv d_npatch4;
@@ -483,6 +485,14 @@ __device__ __forceinline__ int stage_input(float *sm, const Geom &g, const int *
     return 2;
 }
 
+// Zero the haloed arrays, the weight table and the output image; the prefetch ring and its barriers, which
+// the first bulk copies may already be writing, are left alone.
+__device__ __forceinline__ void zero_fill(float *sm, const Geom &g) {
+    float4 *v = reinterpret_cast<float4 *>(sm);
+    for (int i = threadIdx.x; i < g.raw_off / 4; i += blockDim.x) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = g.out_off / 4 + threadIdx.x; i < g.bar_off / 4; i += blockDim.x) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // Issue the bulk copy of one unit's planes into the raw buffer (one thread); a second tensor (grad_out) goes
 // right behind the first on the same barrier.
 template <typename T>
@@ -494,6 +504,20 @@ __device__ __forceinline__ void issue_unit_copies(unsigned long long *bar, char 
     const size_t po = ((size_t)b * g.C + c0) * g.H * g.W;
     bulk_g2s(raw, src + po, bytes, bar);
     if (src2) bulk_g2s(raw + bytes, src2 + po, bytes, bar);
+}
+
+// Start of a block: one thread arms the ring's barriers and sends the first `nstage` units on their way, so
+// that the DRAM round trip runs behind the zero fill, the descriptor set-up and the weight table.
+template <typename T>
+__device__ __forceinline__ void start_prefetch(unsigned long long *bar, char *raw, const Geom &g, const T *__restrict__ src,
+                                               const T *__restrict__ src2, int u_begin, int u_end) {
+    if (threadIdx.x != 0) return;
+    for (int s = 0; s < g.nstage; ++s) mbar_init(bar + s, 1);
+    fence_async_smem();
+    for (int s = 0; s < g.nstage && u_begin + s < u_end; ++s) {
+        const int cgs = (u_begin + s) / g.B;
+        issue_unit_copies<T>(bar + s, raw + s * g.stage_bytes, g, src, src2, cgs * g.NPL, u_begin + s - cgs * g.B);
+    }
 }
 
 // Level l >= 2 from the raw LL band of level l-1 (already in shared memory).  Reads one element past
@@ -687,18 +711,21 @@ __global__ void __launch_bounds__(MAXT, MINB)
 plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0,
                  const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
                  const float *__restrict__ sl, T *__restrict__ out, int *__restrict__ status) {
+    WT_TICK_INIT
     extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
     float *wtab = sm + g.wtab_off;
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sm + g.bar_off);
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
+    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
+    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
+    if (g.bulk) start_prefetch<T>(bar, raw, g, x, nullptr, u_begin, u_end);
+    zero_fill(sm, g);
     unsigned parity = 0;
+    int ring = 0;  // ring entry the current unit arrives in
     const int L = g.L, nlv = g.lvl_start[L + 1];
     const int nlevel_items = g.NPL * nlv, nitems = nlevel_items + g.NPL * g.nbase;
     const size_t HW = (size_t)g.H * g.W;
-    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
-    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
     int c_prev = -1;
     // Staging order: the threads that hold a base tile (the last `nbase_thr` items of the list) are busy with
     // the synthesis of the previous unit when the next one is staged, so the others stage, two patches each
@@ -725,14 +752,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
     PatchD patch1 = decode_patch(g, g.offA, hoist_patch && srank < nstagers ? srank + nstagers : 0x3fffffff);
     __syncthreads();
-    if (g.bulk && tid == 0) {
-        mbar_init(bar, 1);
-        fence_async_smem();
-        const int cg0 = u_begin / g.B;
-        issue_unit_copies<T>(bar, raw, g, x, nullptr, cg0 * g.NPL, u_begin - cg0 * g.B);
-    }
-    __syncthreads();
-    WT_TICK_INIT
+    WT_TICK(9);
     for (int u = u_begin; u < u_end; ++u) {
         const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
         const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
@@ -746,15 +766,15 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         if (g.bulk) {
             // every thread polls the copy barrier itself (bounded); a copy that never lands is flagged and
             // the block carries on with whatever is in the buffer rather than waiting for ever
-            if (!mbar_wait(bar, parity)) atomicExch(status, 1);
-            parity ^= 1u;
+            if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
             WT_TICK(8);
+            const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
             if (hoist_patch) {
-                run_patch<T, true>(sm, g, patch0, reinterpret_cast<const T *>(raw), nvalid);
-                run_patch<T, true>(sm, g, patch1, reinterpret_cast<const T *>(raw), nvalid);
+                run_patch<T, true>(sm, g, patch0, rx, nvalid);
+                run_patch<T, true>(sm, g, patch1, rx, nvalid);
                 lnext = 3;
             } else {
-                lnext = stage_input<T, true>(sm, g, g.offA, reinterpret_cast<const T *>(raw), c, b, srank, nstagers);
+                lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, srank, nstagers);
             }
         } else if (hoist_patch) {
             const T *gsrc = x + ((size_t)b * g.C + c) * HW;
@@ -766,10 +786,15 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         }
         WT_TICK(2);
         __syncthreads();
-        if (g.bulk && tid == 0 && u + 1 < u_end) {  // the raw buffer is free again: fetch the next unit behind the math
-            fence_async_smem();
-            const int cgn = (u + 1) / g.B;
-            issue_unit_copies<T>(bar, raw, g, x, nullptr, cgn * g.NPL, (u + 1) - cgn * g.B);
+        if (g.bulk) {
+            // this ring entry is free again: refill it with the unit `nstage` ahead, behind the math
+            if (tid == 0 && u + g.nstage < u_end) {
+                fence_async_smem();
+                const int cgn = (u + g.nstage) / g.B;
+                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, nullptr, cgn * g.NPL,
+                                     (u + g.nstage) - cgn * g.B);
+            }
+            if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
         }
         WT_TICK(3);
         for (int l = lnext; l <= L; ++l) {
@@ -817,9 +842,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         if (has_base) {
             const float *S = sm + bslot * g.slot_stride;
 #pragma unroll
-#ifndef WT_ABL_NOSYNTH
             for (int hb = 0; hb < TH / 4; ++hb) synth_block(S, g, (TH / 4) * tyy + hb, txx, bias, &acc[4 * hb]);
-#endif
             if (bslot < nvalid) store_tile<T, TH>(g, sm, out + ((size_t)b * g.C + c + bslot) * HW, bslot, tyy, txx, acc);
         }
         if (g.bulk_out) {  // the unit is contiguous in global memory: one bulk store once every tile is in place
@@ -847,9 +870,12 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
                    int *__restrict__ status) {
     extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sm + g.bar_off);
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
+    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
+    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
+    if (g.bulk) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
+    zero_fill(sm, g);
     const int arrays_floats = g.raw_off;  // haloed arrays (and reduction scratch) end where the raw buffer starts
     unsigned parity = 0;
     const int L = g.L, ncls = 1 + 4 * L;
@@ -864,24 +890,15 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     float acc[KK], gsum = 0.f;
 #pragma unroll
     for (int t = 0; t < KK; ++t) acc[t] = 0.f;
-    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
-    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    __syncthreads();
-    if (g.bulk && tid == 0) {
-        mbar_init(bar, 1);
-        fence_async_smem();
-        const int cg0 = u_begin / g.B;
-        issue_unit_copies<T>(bar, raw, g, x, go, cg0 * g.NPL, u_begin - cg0 * g.B);
-    }
+    int ring = 0;
     __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
         const int c = fdiv(u, g.d_B), b = u - c * g.B;  // this kernel is planned with one plane per unit: group = channel
         int lnext;
         if (g.bulk) {
-            if (!mbar_wait(bar, parity)) atomicExch(status, 1);
-            parity ^= 1u;
-            const T *rx = reinterpret_cast<const T *>(raw);
-            const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.plane_bytes);
+            if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
+            const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
+            const T *rg = reinterpret_cast<const T *>(raw + ring * g.stage_bytes + (size_t)g.NPL * g.plane_bytes);
             lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, tid, nthr);
             stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
         } else {
@@ -889,10 +906,14 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
         }
         __syncthreads();
-        if (g.bulk && tid == 0 && u + 1 < u_end) {
-            fence_async_smem();
-            const int cgn = (u + 1) / g.B;
-            issue_unit_copies<T>(bar, raw, g, x, go, cgn * g.NPL, (u + 1) - cgn * g.B);
+        if (g.bulk) {
+            if (tid == 0 && u + g.nstage < u_end) {
+                fence_async_smem();
+                const int cgn = (u + g.nstage) / g.B;
+                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, go, cgn * g.NPL,
+                                     (u + g.nstage) - cgn * g.B);
+            }
+            if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
         }
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
@@ -989,16 +1010,17 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                  float *__restrict__ partl /* level l at l*C*np*100 */, int *__restrict__ status) {
     extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int i = tid; i < g.smem_floats; i += nthr) sm[i] = 0.f;
     float *wtab = sm + g.wtab_off;
     unsigned long long *bar = reinterpret_cast<unsigned long long *>(sm + g.bar_off);
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
+    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
+    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
+    if (BULK) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
+    zero_fill(sm, g);
     unsigned parity = 0;
     const int L = g.L, nlv = g.lvl_start[L + 1], ncls = 1 + 4 * L;
     const int nlevel_items = g.NPL * nlv, nitems = nlevel_items + g.NPL * g.nbase;
     const size_t HW = (size_t)g.H * g.W;
-    const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
-    const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
     int bslot = 0, tyy = 0, txx = 0;
     bool has_base = false;
     const ItemD item = decode_item(g, tid, nlevel_items, nitems, bslot, tyy, txx, has_base);
@@ -1011,13 +1033,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
     for (int t = 0; t < KK; ++t) accw[t] = 0.f;
     int c_prev = -1;
-    __syncthreads();
-    if (BULK && tid == 0) {
-        mbar_init(bar, 1);
-        fence_async_smem();
-        const int cg0 = u_begin / g.B;
-        issue_unit_copies<T>(bar, raw, g, x, go, cg0 * g.NPL, u_begin - cg0 * g.B);
-    }
+    int ring = 0;
     __syncthreads();
     for (int u = u_begin; u < u_end; ++u) {
         const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
@@ -1028,10 +1044,9 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         }
         int lnext;
         if (BULK) {
-            if (!mbar_wait(bar, parity)) atomicExch(status, 1);
-            parity ^= 1u;
-            const T *rx = reinterpret_cast<const T *>(raw);
-            const T *rg = reinterpret_cast<const T *>(raw + (size_t)g.NPL * g.plane_bytes);
+            if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
+            const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
+            const T *rg = reinterpret_cast<const T *>(raw + ring * g.stage_bytes + (size_t)g.NPL * g.plane_bytes);
             if (hoist_patch) {
                 run_patch<T, true>(sm, g, patch0, rx, nvalid);
                 run_patch<T, true>(sm, g, patch0, rg, nvalid, dA0, dA1, dA2);
@@ -1054,10 +1069,14 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
         }
         __syncthreads();
-        if (BULK && tid == 0 && u + 1 < u_end) {
-            fence_async_smem();
-            const int cgn = (u + 1) / g.B;
-            issue_unit_copies<T>(bar, raw, g, x, go, cgn * g.NPL, (u + 1) - cgn * g.B);
+        if (BULK) {
+            if (tid == 0 && u + g.nstage < u_end) {
+                fence_async_smem();
+                const int cgn = (u + g.nstage) / g.B;
+                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, go, cgn * g.NPL,
+                                     (u + g.nstage) - cgn * g.B);
+            }
+            if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
         }
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
@@ -1205,20 +1224,42 @@ inline void fill_common(Geom &g, int B, int C, int H, int W, int L, int elem_byt
     g.raw_slot_bytes = g.plane_bytes;
 }
 
-// Tail of the shared-memory layout: [arrays][weight table][raw planes (bulk only)][mbarrier].  Returns floats.
-inline long long finish_layout(Geom &g, long long arrays_floats, int wtab_floats, int raw_tensors, bool use_bulk) {
+// Tail of the shared-memory layout: [arrays][weight table][ring of raw units (bulk only)][output image]
+// [mbarriers].  Returns floats.
+inline long long finish_layout(Geom &g, long long arrays_floats, int wtab_floats, int raw_tensors, bool use_bulk,
+                               int nstage = 1) {
     long long off = pad4((int)arrays_floats);
     g.wtab_off = (int)off;
     off += pad4(wtab_floats);
     g.raw_off = (int)off;
-    if (use_bulk) off += ((long long)raw_tensors * g.NPL * g.plane_bytes + 3) / 4;
+    g.nstage = use_bulk ? nstage : 1;
+    g.stage_bytes = raw_tensors * g.NPL * g.plane_bytes;  // a multiple of 16 whenever bulk copies are allowed
+    if (use_bulk) off += ((long long)g.nstage * g.stage_bytes + 3) / 4;
     off = pad4((int)off);
     g.out_off = (int)off;
     g.bulk_out = (use_bulk && !g.vec) ? 1 : 0;  // rows that are not 16-byte multiples: assemble the unit on chip
     if (g.bulk_out) off += ((long long)g.NPL * g.plane_bytes + 3) / 4;
     off = pad4((int)off);
     g.bar_off = (int)off;
-    return off + 4;
+    return off + 2 * MAX_STAGES;
+}
+
+// Deepen the prefetch ring of a finished plan as far as the shared memory left beside its resident blocks
+// allows: short units (small planes) finish faster than one DRAM round trip, so one unit of look-ahead
+// leaves the block waiting for its copy.
+inline void deepen_prefetch(Geom &g) {
+    if (!g.bulk) return;
+    // the layout up to the ring is kept: [0, wtab_off) arrays, [wtab_off, raw_off) weight table
+    const int raw_tensors = g.stage_bytes / (g.NPL * g.plane_bytes);
+    for (int ns = 2; ns <= MAX_STAGES; ++ns) {
+        if ((long long)(ns - 1) * g.nblocks >= g.units) break;  // deeper than the units a block has
+        Geom t = g;
+        const long long fl = finish_layout(t, g.wtab_off, g.raw_off - g.wtab_off, raw_tensors, true, ns);
+        const long long bytes = fl * 4;
+        if (bytes > SMEM_LIMIT || (long long)g.blocks_per_sm * (bytes + 1024) > SMEM_PER_SM) break;
+        t.smem_floats = (int)fl;
+        g = t;
+    }
 }
 
 // Slot layout; returns floats per slot.  with_g: second copy of the input pyramid (grad_out); with_z:
@@ -1448,6 +1489,7 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
     bool ok = false;
     if (!((tune >> 23) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 8);
     if (!((tune >> 22) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    if (ok) deepen_prefetch(best);
     return ok;
 }
 inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
@@ -1455,6 +1497,7 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
     bool ok = false;
     if (!((tune >> 23) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 8);
     if (!((tune >> 22) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    if (ok) deepen_prefetch(best);
     return ok;
 }
 inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
@@ -1463,6 +1506,7 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
     bool ok = false;
     if (!((tune >> 23) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 8);
     if (!((tune >> 22) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 4);
+    if (ok) deepen_prefetch(best);
     return ok;
 }
 

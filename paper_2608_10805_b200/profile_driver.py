@@ -1,6 +1,6 @@
 """Small driver for profiler captures: runs forward+backward of a named workload (optionally with a smaller
 batch) a few times through the C ABI on random tensors.  Usage:
-    python -m paper_2608_10805_b200.profile_driver <workload> [batch] [repeats]
+    python -m paper_2608_10805_b200.profile_driver <workload> [batch] [repeats] [flags]
 """
 import sys
 
@@ -16,8 +16,9 @@ def main():
     if len(sys.argv) > 2:
         wl = wl.with_(B=int(sys.argv[2]))
     reps = int(sys.argv[3]) if len(sys.argv) > 3 else 2
+    flags = int(sys.argv[4], 0) if len(sys.argv) > 4 else 0
     tdt = wt.DTYPE_NAMES[wl.dtype]
-    desc = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, tdt)
+    desc = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, tdt, flags)
     x = torch.randn(wl.B, wl.C, wl.H, wl.W, device="cuda").to(tdt)
     g = torch.randn_like(x)
     w0 = torch.randn(wl.C, wl.k, wl.k, device="cuda") * 0.1
