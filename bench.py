@@ -31,7 +31,10 @@ FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FP32 lanes x 2 FL
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (bytes; keyed by workload and kernel).  None where no capture exists.
-NCU_DRAM_TRAFFIC = {}
+NCU_DRAM_TRAFFIC = {
+    ("stage1_f32", "plane_bwd_kernel"): 154784768 + 49147648,
+    ("stage1_f32", "plane_fwd_kernel"): 77334528 + 32297984,
+}
 
 
 def load_measured_peaks():
@@ -296,7 +299,8 @@ def main():
                      "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 FLOP x 1.965 GHz (measured 74.1 with a packed-FMA loop)",
                      "launch_ms": dom_ms, "flops_per_launch": dom_fl,
                      "forward_kernel": {"launch_ms": fwd_kernel_ms, "achieved": fl_fwd / (fwd_kernel_ms * 1e-3) / 1e12,
-                                        "frac": fl_fwd / (fwd_kernel_ms * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS}},
+                                        "frac": fl_fwd / (fwd_kernel_ms * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS,
+                                        "traffic": NCU_DRAM_TRAFFIC.get((wl.name, "plane_fwd_kernel"))}},
         "step_rooflines": {
             "alu_frac": fl_step / (ms_step * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS,
             "hbm_compulsory_gbs": hbm_step / (ms_step * 1e-3) / 1e9,
