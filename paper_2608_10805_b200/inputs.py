@@ -45,6 +45,14 @@ WORKLOADS = {
     "stage2_bf16": Workload("stage2_bf16", 128, 192, 28, 28, 5, 2, "bf16", 3),
     "stage3_bf16": Workload("stage3_bf16", 128, 384, 14, 14, 5, 1, "bf16", 3),
     "stage4_bf16": Workload("stage4_bf16", 128, 768, 7, 7, 5, 1, "bf16", 3),
+    # the network's own depth schedule, L = (5, 4, 3, 2) on the four stages: repeated odd padding 7 -> 4 -> 2
+    "convnext_s1_bf16": Workload("convnext_s1_bf16", 64, 96, 56, 56, 5, 5, "bf16", 5),
+    "convnext_s2_bf16": Workload("convnext_s2_bf16", 64, 192, 28, 28, 5, 4, "bf16", 5),
+    "convnext_s3_bf16": Workload("convnext_s3_bf16", 64, 384, 14, 14, 5, 3, "bf16", 5),
+    "convnext_s4_bf16": Workload("convnext_s4_bf16", 64, 768, 7, 7, 5, 2, "bf16", 5),
+    # kernel-size variants of the stage-1 layer
+    "stage1_k3_f32": Workload("stage1_k3_f32", 16, 96, 56, 56, 3, 3, "f32", 6),
+    "stage1_k7_f32": Workload("stage1_k7_f32", 16, 96, 56, 56, 7, 3, "f32", 6),
     "large_f16": Workload("large_f16", 16, 256, 256, 256, 5, 5, "f16", 4),
     "large_odd_f16": Workload("large_odd_f16", 16, 256, 225, 225, 5, 5, "f16", 4),
 }

@@ -65,6 +65,19 @@ def test_wtconvnext_stage_set_bf16(name):
     _run_full_and_compare(wl, [0, 1, wl.C // 2, wl.C - 2, wl.C - 1])
 
 
+@pytest.mark.parametrize("name", ["convnext_s1_bf16", "convnext_s2_bf16", "convnext_s3_bf16", "convnext_s4_bf16"])
+def test_wtconvnext_depth_schedule_bf16(name):
+    wl = inputs.WORKLOADS[name]  # L = (5, 4, 3, 2): grids shrink through odd sizes (7 -> 4 -> 2, 14 -> 7 -> 4 -> 2)
+    assert wt.wtconv_plan_name(wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wt.DTYPE_NAMES[wl.dtype])) == "plane"
+    _run_full_and_compare(wl, [0, 1, wl.C // 2, wl.C - 1])
+
+
+@pytest.mark.parametrize("name", ["stage1_k3_f32", "stage1_k7_f32"])
+def test_kernel_size_variants(name):
+    wl = inputs.WORKLOADS[name]
+    _run_full_and_compare(wl, [0, wl.C // 2, wl.C - 1])
+
+
 @pytest.mark.parametrize("dtype", ["f32", "f16"])
 @pytest.mark.parametrize("L", [1, 2, 3, 4, 5])
 def test_level_sweep(L, dtype):

@@ -30,6 +30,9 @@ SMALL = [
     Workload("stage4_small", 3, 5, 7, 7, 5, 1, "f32", 22),
     Workload("sweep_small_L5", 1, 3, 64, 64, 5, 5, "f32", 23),
     Workload("big_plane", 1, 2, 225, 225, 5, 5, "f32", 24),
+    Workload("convnext_s1_small", 2, 3, 56, 56, 5, 5, "f32", 25),   # the network's depth schedule L = (5, 4, 3, 2)
+    Workload("convnext_s2_small", 2, 3, 28, 28, 5, 4, "f32", 26),
+    Workload("convnext_s3_small", 3, 5, 14, 14, 5, 3, "f32", 27),
 ]
 
 
