@@ -1002,7 +1002,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 //                    closed-form synthesis of Proposition 2 and the store of grad_x.
 // Used when a unit's item list fits one round of the block (<= 256 tiles); otherwise the separate weight-
 // gradient and input-gradient kernels run.
-template <typename T, int TH, bool BULK>
+template <typename T, int TH, int BULK>  // BULK: tensors prefetched by bulk copy (0 none, 1 x only, 2 x and grad_out)
 __global__ void __launch_bounds__(256, 2)
 plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                  const float *__restrict__ w0, const float *__restrict__ s0, const float *__restrict__ wl,
@@ -1015,7 +1015,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    if (BULK) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
+    if (BULK) start_prefetch<T>(bar, raw, g, x, BULK == 2 ? go : nullptr, u_begin, u_end);
     zero_fill(sm, g);
     unsigned parity = 0;
     const int L = g.L, nlv = g.lvl_start[L + 1], ncls = 1 + 4 * L;
@@ -1047,15 +1047,22 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
             const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
             const T *rg = reinterpret_cast<const T *>(raw + ring * g.stage_bytes + (size_t)g.NPL * g.plane_bytes);
+            const T *gg = go + ((size_t)b * g.C + c) * HW;  // grad_out straight from global memory when BULK == 1
             if (hoist_patch) {
+                // the global loads of grad_out go first so that their latency runs behind the x patches
+                if (BULK == 1) {
+                    run_patch<T, false>(sm, g, patch0, gg, nvalid, dA0, dA1, dA2);
+                    run_patch<T, false>(sm, g, patch1, gg, nvalid, dA0, dA1, dA2);
+                }
                 run_patch<T, true>(sm, g, patch0, rx, nvalid);
-                run_patch<T, true>(sm, g, patch0, rg, nvalid, dA0, dA1, dA2);
+                if (BULK == 2) run_patch<T, true>(sm, g, patch0, rg, nvalid, dA0, dA1, dA2);
                 run_patch<T, true>(sm, g, patch1, rx, nvalid);
-                run_patch<T, true>(sm, g, patch1, rg, nvalid, dA0, dA1, dA2);
+                if (BULK == 2) run_patch<T, true>(sm, g, patch1, rg, nvalid, dA0, dA1, dA2);
                 lnext = 3;
             } else {
                 lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, tid, nthr);
-                stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
+                if (BULK == 2) stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
+                else stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
             }
         } else if (hoist_patch) {
             const size_t po = ((size_t)b * g.C + c) * HW;
@@ -1073,7 +1080,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             if (tid == 0 && u + g.nstage < u_end) {
                 fence_async_smem();
                 const int cgn = (u + g.nstage) / g.B;
-                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, go, cgn * g.NPL,
+                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, BULK == 2 ? go : nullptr, cgn * g.NPL,
                                      (u + g.nstage) - cgn * g.B);
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
@@ -1103,11 +1110,16 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) gsum += d[rr][cc];
                 }
+                // the next window row is fetched while the current one is used
+                float4 n0 = *reinterpret_cast<const float4 *>(ysrc);
+                float4 n1 = *reinterpret_cast<const float4 *>(ysrc + 4);
 #pragma unroll
                 for (int rr = 0; rr < TH + 4; ++rr) {
-                    const float4 q0 = *reinterpret_cast<const float4 *>(ysrc + rr * pitch);
-                    const float4 q1 = *reinterpret_cast<const float4 *>(ysrc + rr * pitch + 4);
-                    const float in[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+                    const float in[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+                    if (rr + 1 < TH + 4) {
+                        n0 = *reinterpret_cast<const float4 *>(ysrc + (rr + 1) * pitch);
+                        n1 = *reinterpret_cast<const float4 *>(ysrc + (rr + 1) * pitch + 4);
+                    }
 #pragma unroll
                     for (int uu = 0; uu < 5; ++uu) {
                         const int dr = rr - uu;
@@ -1443,10 +1455,12 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
         if (scratch > arrays) arrays = scratch;
         const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 20) & 1);
         bool any = false;
-        for (int use_bulk = can_bulk ? 1 : 0; use_bulk >= 0; --use_bulk) {
+        // use_bulk = tensors that arrive by bulk copy: both or none (x only, with grad_out read by plain loads,
+        // is built into the kernel as BULK == 1 but measured slower than no prefetch at 56 x 56 fp32)
+        for (int use_bulk = can_bulk ? 2 : 0; use_bulk >= 0; use_bulk -= 2) {
         Geom cg = g;
         cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
-        const long long smem_floats = finish_layout(cg, arrays, wtab, 2, use_bulk);
+        const long long smem_floats = finish_layout(cg, arrays, wtab, use_bulk ? use_bulk : 1, use_bulk > 0);
         const long long bytes = smem_floats * 4;
         if (bytes > SMEM_LIMIT) continue;
         any = true;
@@ -1460,7 +1474,8 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
             double occ = (double)bps * T / 512.0;
             if (occ > 1.0) occ = 1.0;
             const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
-            const double sc = teff * ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.85) *
+            const double sc = teff * ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap *
+                              (use_bulk == 2 ? 1.0 : (use_bulk == 1 ? 0.93 : 0.85)) *
                               partition_eff(units, nblocks) * ((double)C / ((double)ngroups * npl));
             if (sc > best.score + 1e-9) {
                 best = cg;
@@ -1583,9 +1598,9 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
                                                                          reinterpret_cast<int *>(ws));     \
     }
         if (gw.th == 8) {
-            if (gw.bulk) WT_LAUNCH_BWD(8, true) else WT_LAUNCH_BWD(8, false)
+            if (gw.bulk == 2) WT_LAUNCH_BWD(8, 2) else if (gw.bulk == 1) WT_LAUNCH_BWD(8, 1) else WT_LAUNCH_BWD(8, 0)
         } else {
-            if (gw.bulk) WT_LAUNCH_BWD(4, true) else WT_LAUNCH_BWD(4, false)
+            if (gw.bulk == 2) WT_LAUNCH_BWD(4, 2) else if (gw.bulk == 1) WT_LAUNCH_BWD(4, 1) else WT_LAUNCH_BWD(4, 0)
         }
 #undef WT_LAUNCH_BWD
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
