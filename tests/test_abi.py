@@ -81,6 +81,29 @@ def test_plan_and_launch_count(lib):
     assert wt.wtconv_plan_name(dt) == "tiled"
 
 
+def test_scratch_memory_accounting(lib):
+    """Device memory the layer needs beyond its inputs and outputs.  Whole-plane kernels keep every intermediate
+    on chip: the forward needs only a status word and the backward its per-block gradient partials, a few
+    MiB at most on every stage of the network (they fit the library's built-in scratch).  The tiled path keeps
+    Z^l and the raw carriers in HBM: 4 + 1 float32 per level-l coefficient and plane (the carrier of the last level is not needed)."""
+    from paper_2608_10805_b200 import inputs
+    for name in ("stage1_f32", "stage1_bf16", "stage2_bf16", "stage3_bf16", "stage4_bf16",
+                 "convnext_s1_bf16", "convnext_s2_bf16", "convnext_s3_bf16", "convnext_s4_bf16"):
+        wl = inputs.WORKLOADS[name]
+        d = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wl.dtype)
+        assert wt.wtconv_plan_name(d) == "plane"
+        fb, bb = wt.wtconv_workspace_bytes(d)
+        assert fb == 256 and bb < (8 << 20), (name, fb, bb)
+    wl = inputs.WORKLOADS["large_f16"]
+    d = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wl.dtype)
+    fb, _ = wt.wtconv_workspace_bytes(d)
+    P, coeffs = wl.B * wl.C, 0
+    for l in range(1, wl.L + 1):
+        Hl, Wl = wt.wtconv_level_shape(d, l)
+        coeffs += (4 + (1 if l < wl.L else 0)) * Hl * Wl
+    assert abs(fb - 4 * P * coeffs) <= 4096 * (wl.L + 2), (fb, 4 * P * coeffs)
+
+
 def test_binding_refuses_to_run_without_the_library(monkeypatch):
     monkeypatch.setattr(wt, "_lib", None)
     monkeypatch.setattr(wt, "LIB_PATH", "/nonexistent/libwtconv_b200.so")
