@@ -5,41 +5,71 @@
 // the weights when they are loaded (Eq. 8), and the synthesis is the single bit-indexed pass of
 // Proposition 2 with the base convolution fused into the final store (Sec. 4.2).
 //
-// Thread layout of every kernel here: 256 threads = 8 warps; lane = column inside a 32-wide
-// tile.  In the level kernels warp w owns subband (w & 3) and the upper or lower half (w >> 2)
-// of a 16-row coefficient tile, so a thread only ever sees one subband and can keep that
-// subband's k*k weights and k*k weight-gradient accumulators in registers across a whole
-// batch loop.
+// Thread layout of every kernel here: 256 threads, a 4 x 4 block of outputs per thread (register tile, window
+// rows read as aligned float4 loads).  In the level kernels 64 threads own each subband of a 32 x 32
+// coefficient tile, so a thread only ever sees one subband and can keep that subband's k*k weights and k*k
+// weight-gradient accumulators in registers across a whole batch loop; the synthesis kernels work on
+// 64 x 64 pixel tiles.
 #pragma once
 #include "common.cuh"
 
 namespace wt {
 namespace tiled {
 
-constexpr int TW = 32;       // tile width (coefficients or pixels)
-constexpr int TH = 16;       // tile height
+constexpr int TW = 32;       // level kernels: tile width in coefficients
+constexpr int TH = 32;       // level kernels: tile height in coefficients
 constexpr int NTHREADS = 256;
-constexpr int ROWS_PER_THREAD = 8;  // level kernels: TH / 2 halves
+
+// Shared-memory tile of TWc x THc outputs with halo R = K/2.  Every thread computes a 4 x 4 output block; its
+// window starts at a multiple of four floats, so window rows are read as NQ aligned float4 loads, and the pitch
+// P leaves room for the last thread's last load.
+template <int K, int TWc, int THc> struct TileDims {
+    static constexpr int R = K / 2;
+    static constexpr int NQ = (4 + K - 1 + 3) / 4;
+    static constexpr int W = TWc + 2 * R, H = THc + 2 * R;
+    static constexpr int P = TWc - 4 + 4 * NQ;
+};
+template <int K> using LevelTile = TileDims<K, TW, TH>;
+
+// Two horizontally adjacent activations as floats (the pair starts at an even column of an even-length row, so
+// it is aligned to its own size).
+__device__ __forceinline__ float2 load_pair(const float *p) { return __ldg(reinterpret_cast<const float2 *>(p)); }
+__device__ __forceinline__ float2 load_pair(const __half *p) {
+    const unsigned q = __ldg(reinterpret_cast<const unsigned *>(p));
+    return __half22float2(*reinterpret_cast<const __half2 *>(&q));
+}
+__device__ __forceinline__ float2 load_pair(const __nv_bfloat16 *p) {
+    const unsigned q = __ldg(reinterpret_cast<const unsigned *>(p));
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q));
+}
 
 // Stage the four subbands of the level grid (Hl x Wl) around tile origin (i0, j0), with halo R,
 // from the previous carrier plane `xp` (Hp x Wp).  Positions outside the level grid are zero
 // (the depthwise conv's zero padding); pixels outside the carrier are zero (odd-size padding).
 template <typename Tin, int K>
 __device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int Hp, int Wp, int Hl, int Wl, int i0,
-                                               int j0, float (*Ys)[TH + K - 1][TW + K] /* [4] */) {
-    constexpr int R = K / 2, SW = TW + 2 * R, SH = TH + 2 * R;
-    for (int e = threadIdx.x; e < SH * SW; e += NTHREADS) {
-        int li = e / SW, lj = e - li * SW;
-        int i = i0 + li - R, j = j0 + lj - R;
+                                               int j0, float (*Ys)[LevelTile<K>::H][LevelTile<K>::P] /* [4] */) {
+    using D = LevelTile<K>;
+    const bool even = (Wp & 1) == 0;
+    for (int e = threadIdx.x; e < D::H * D::P; e += NTHREADS) {
+        const int li = e / D::P, lj = e - li * D::P;
+        const int i = i0 + li - D::R, j = j0 + lj - D::R;
         Haar4 h = {0.f, 0.f, 0.f, 0.f};
-        if (i >= 0 && i < Hl && j >= 0 && j < Wl) {
-            int y = 2 * i, x = 2 * j;
-            bool x1 = (x + 1 < Wp), y1 = (y + 1 < Hp);
+        if (lj < D::W && i >= 0 && i < Hl && j >= 0 && j < Wl) {
+            const int y = 2 * i, x = 2 * j;
+            const bool y1 = (y + 1 < Hp);
             const Tin *q = xp + (size_t)y * Wp + x;
-            float a = ldf(q);
-            float b = x1 ? ldf(q + 1) : 0.f;
-            float c = y1 ? ldf(q + Wp) : 0.f;
-            float d = (x1 && y1) ? ldf(q + Wp + 1) : 0.f;
+            float a, b, c = 0.f, d = 0.f;
+            if (even) {
+                const float2 t = load_pair(q);
+                a = t.x; b = t.y;
+                if (y1) { const float2 u = load_pair(q + Wp); c = u.x; d = u.y; }
+            } else {
+                const bool x1 = (x + 1 < Wp);
+                a = ldf(q);
+                b = x1 ? ldf(q + 1) : 0.f;
+                if (y1) { c = ldf(q + Wp); d = x1 ? ldf(q + Wp + 1) : 0.f; }
+            }
             h = haar_butterfly(a, b, c, d);
         }
         Ys[0][li][lj] = h.ll;
@@ -49,24 +79,71 @@ __device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int H
     }
 }
 
-// Column conv: 8 vertically adjacent outputs at column `lx` (tile coords, halo-shifted), rows
-// r0..r0+7, of S (one subband, with halo) against register weights w[K*K].
-template <int K>
-__device__ __forceinline__ void column_conv(const float (*S)[TW + K], int r0, int lx, const float *w, float *acc) {
+// 4 x 4 outputs of the k x k correlation with register weights; `Xs` has pitch P and the window starts at
+// (ly0, lx0), lx0 a multiple of 4, so its rows come as aligned float4 loads.
+template <int K, int P>
+__device__ __forceinline__ void block_conv(const float (*Xs)[P], int ly0, int lx0, const float *w, float (&acc)[4][4]) {
+    constexpr int NQ = (4 + K - 1 + 3) / 4;
 #pragma unroll
-    for (int r = 0; r < ROWS_PER_THREAD; ++r) acc[r] = 0.f;
+    for (int rr = 0; rr < 4 + K - 1; ++rr) {
+        float in[4 * NQ];
 #pragma unroll
-    for (int rr = 0; rr < ROWS_PER_THREAD + K - 1; ++rr) {
-        float in[K];
-#pragma unroll
-        for (int v = 0; v < K; ++v) in[v] = S[r0 + rr][lx + v];
+        for (int q = 0; q < NQ; ++q) {
+            const float4 v = *reinterpret_cast<const float4 *>(&Xs[ly0 + rr][lx0 + 4 * q]);
+            in[4 * q] = v.x; in[4 * q + 1] = v.y; in[4 * q + 2] = v.z; in[4 * q + 3] = v.w;
+        }
 #pragma unroll
         for (int u = 0; u < K; ++u) {
-            int r = rr - u;
-            if (r >= 0 && r < ROWS_PER_THREAD) {
+            const int r = rr - u;
+            if (r >= 0 && r < 4) {
 #pragma unroll
-                for (int v = 0; v < K; ++v) acc[r] = fmaf(w[u * K + v], in[v], acc[r]);
+                for (int v = 0; v < K; ++v)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(w[u * K + v], in[c + v], acc[r][c]);
             }
+        }
+    }
+}
+
+// Weight-gradient taps of a 4 x 4 block: gw[u,v] += sum_{r,c} d[r][c] * Xs[ly0 + r + u][lx0 + c + v].
+template <int K, int P>
+__device__ __forceinline__ void block_wgrad(const float (*Xs)[P], int ly0, int lx0, const float (&d)[4][4], float *gw) {
+    constexpr int NQ = (4 + K - 1 + 3) / 4;
+#pragma unroll
+    for (int rr = 0; rr < 4 + K - 1; ++rr) {
+        float in[4 * NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            const float4 v = *reinterpret_cast<const float4 *>(&Xs[ly0 + rr][lx0 + 4 * q]);
+            in[4 * q] = v.x; in[4 * q + 1] = v.y; in[4 * q + 2] = v.z; in[4 * q + 3] = v.w;
+        }
+#pragma unroll
+        for (int u = 0; u < K; ++u) {
+            const int r = rr - u;
+            if (r >= 0 && r < 4) {
+#pragma unroll
+                for (int v = 0; v < K; ++v)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) gw[u * K + v] = fmaf(d[r][c], in[c + v], gw[u * K + v]);
+            }
+        }
+    }
+}
+
+// Store rows of four fp32 coefficients of a level grid (vector store where the row length allows).
+__device__ __forceinline__ void store_coeff_block(float *__restrict__ plane, int Hl, int Wl, int I0, int J0,
+                                                  const float (&a)[4][4]) {
+    const bool vec = (Wl & 3) == 0 && J0 + 3 < Wl;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        if (I0 + r >= Hl) break;
+        float *q = plane + (size_t)(I0 + r) * Wl + J0;
+        if (vec) {
+            *reinterpret_cast<float4 *>(q) = make_float4(a[r][0], a[r][1], a[r][2], a[r][3]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (J0 + c < Wl) q[c] = a[r][c];
         }
     }
 }
@@ -79,85 +156,216 @@ __global__ void __launch_bounds__(NTHREADS)
 level_fwd_kernel(const Tin *__restrict__ Xprev, int Hp, int Wp, int Hl, int Wl, int C,
                  const float *__restrict__ w /* [C][4][K][K] */, const float *__restrict__ s /* [C][4] */,
                  float *__restrict__ Z /* [P][4][Hl][Wl] */, float *__restrict__ Xl /* [P][Hl][Wl] or null */) {
-    constexpr int R = K / 2;
-    __shared__ float Ys[4][TH + K - 1][TW + K];
+    using D = LevelTile<K>;
+    constexpr int KK = K * K;
+    __shared__ __align__(16) float Ys[4][D::H][D::P];
+    __shared__ float Ws[4][KK];
     const int p = blockIdx.x, c = p % C;
     const int j0 = blockIdx.y * TW, i0 = blockIdx.z * TH;
     stage_subbands<Tin, K>(Xprev + (size_t)p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int sub = warp & 3, r0 = (warp >> 2) * ROWS_PER_THREAD;
-    float wr[K * K];
-    const float sc = __ldg(s + c * 4 + sub);
-#pragma unroll
-    for (int t = 0; t < K * K; ++t) wr[t] = sc * __ldg(w + ((size_t)c * 4 + sub) * K * K + t);  // Eq. 8
+    if (threadIdx.x < 4 * KK)  // Eq. 8
+        Ws[threadIdx.x / KK][threadIdx.x % KK] = __ldg(s + c * 4 + threadIdx.x / KK) * __ldg(w + (size_t)c * 4 * KK + threadIdx.x);
     __syncthreads();
-    float acc[ROWS_PER_THREAD];
-    column_conv<K>(Ys[sub], r0, lane, wr, acc);
-    const int j = j0 + lane;
-    if (j < Wl) {
-        float *zp = Z + ((size_t)p * 4 + sub) * Hl * Wl;
+    const int sub = threadIdx.x >> 6, tx = threadIdx.x & 7, ty = (threadIdx.x >> 3) & 7;
+    const int I0 = i0 + 4 * ty, J0 = j0 + 4 * tx;
+    if (I0 >= Hl || J0 >= Wl) return;
+    float wr[KK];
 #pragma unroll
-        for (int r = 0; r < ROWS_PER_THREAD; ++r) {
-            int i = i0 + r0 + r;
-            if (i < Hl) {
-                zp[(size_t)i * Wl + j] = acc[r];
-                if (sub == 0 && Xl) Xl[((size_t)p * Hl + i) * Wl + j] = Ys[0][r0 + r + R][lane + R];
-            }
-        }
+    for (int t = 0; t < KK; ++t) wr[t] = Ws[sub][t];
+    float acc[4][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) acc[r][cc] = 0.f;
+    block_conv<K, D::P>(Ys[sub], 4 * ty, 4 * tx, wr, acc);
+    store_coeff_block(Z + ((size_t)p * 4 + sub) * Hl * Wl, Hl, Wl, I0, J0, acc);
+    if (sub == 0 && Xl) {
+        float ll[4][4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) ll[r][cc] = Ys[0][4 * ty + D::R + r][4 * tx + D::R + cc];
+        store_coeff_block(Xl + (size_t)p * Hl * Wl, Hl, Wl, I0, J0, ll);
     }
 }
 
 // ---------------------------------------------------------------------------------------------
 // Forward synthesis kernel: out = Wfold^0 (*) x + bfold + sum_l (Prop. 2 term of Z^l).
-// grid (P, tiles_x, tiles_y); thread = column lane, rows 2*warp, 2*warp+1 of the tile.
+// grid (P, tiles_x, tiles_y) over STW x STH pixel tiles; one 4 x 4 pixel block per thread.
 // ---------------------------------------------------------------------------------------------
 struct LevelPtrs {
     const float *z[8];  // per level l (index l-1): [P][4][Hl][Wl]
     int Hl[8], Wl[8];
 };
 
+// Pixel tile of the synthesis kernels: STW x STH pixels per block, a 4 x 4 pixel block per thread
+// (16 x 16 threads).  The x tile sits in shared memory with halo R and a pitch that keeps every
+// thread's window start 16-byte aligned.
+constexpr int STW = 64, STH = 64;
+template <int K> struct SynthTile : TileDims<K, STW, STH> {
+    static constexpr int XW = TileDims<K, STW, STH>::W, XH = TileDims<K, STW, STH>::H, XP = TileDims<K, STW, STH>::P;
+};
+
+// Four consecutive activations as floats (16-byte / 8-byte aligned vector load).
+__device__ __forceinline__ float4 load_vec4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ float4 load_vec4(const __half *p) {
+    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ float4 load_vec4(const __nv_bfloat16 *p) {
+    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+
+// Stage the STW x STH pixel tile at (y0, x0) of plane `xp` with halo R; zero outside the image.  When the
+// row length is a multiple of 4 the tile's own columns come as vector loads of 4 pixels (they are then
+// either all inside the image or all outside) and only the 2R halo columns go element by element.
+template <typename T, int K>
+__device__ __forceinline__ void stage_pixels(const T *__restrict__ xp, int H, int W, int y0, int x0,
+                                             float (*Xs)[SynthTile<K>::XP]) {
+    using S = SynthTile<K>;
+    if ((W & 3) == 0) {
+        for (int e = threadIdx.x; e < S::XH * (STW / 4); e += NTHREADS) {
+            const int ly = e / (STW / 4), j = e - ly * (STW / 4);
+            const int yy = y0 + ly - S::R, xx = x0 + 4 * j;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (yy >= 0 && yy < H && xx < W) v = load_vec4(xp + (size_t)yy * W + xx);
+            float *q = &Xs[ly][S::R + 4 * j];
+            q[0] = v.x; q[1] = v.y; q[2] = v.z; q[3] = v.w;
+        }
+        for (int e = threadIdx.x; e < S::XH * (S::XP - STW); e += NTHREADS) {
+            const int ly = e / (S::XP - STW), h = e - ly * (S::XP - STW);
+            const int lx = h < S::R ? h : STW + h;  // left halo, then right halo and the pitch padding
+            const int yy = y0 + ly - S::R, xx = x0 + lx - S::R;
+            Xs[ly][lx] = (yy >= 0 && yy < H && xx >= 0 && xx < W) ? ldf(xp + (size_t)yy * W + xx) : 0.f;
+        }
+        return;
+    }
+    for (int e = threadIdx.x; e < S::XH * S::XP; e += NTHREADS) {
+        const int ly = e / S::XP, lx = e - ly * S::XP;
+        const int yy = y0 + ly - S::R, xx = x0 + lx - S::R;
+        Xs[ly][lx] = (yy >= 0 && yy < H && xx >= 0 && xx < W) ? ldf(xp + (size_t)yy * W + xx) : 0.f;
+    }
+}
+
+// Proposition 2 for the 4 x 4 pixel block with origin (Y0, X0), both multiples of 4, of plane p: level 1
+// contributes 2 x 2 coefficients per subband, level 2 one coefficient whose signs vary inside the block, every
+// deeper level one coefficient with a block-wide sign.
+__device__ __forceinline__ void block_synthesis(const LevelPtrs &lv, int L, size_t p, int Y0, int X0, float (&a)[4][4]) {
+    if (L >= 1) {
+        const int Hl = lv.Hl[0], Wl = lv.Wl[0];
+        const size_t S = (size_t)Hl * Wl;
+        const float *zp = lv.z[0] + p * 4 * S;
+#pragma unroll
+        for (int ci = 0; ci < 2; ++ci)
+#pragma unroll
+            for (int cj = 0; cj < 2; ++cj) {
+                const int i = (Y0 >> 1) + ci, j = (X0 >> 1) + cj;
+                if (i < Hl && j < Wl) {
+                    const float *q = zp + (size_t)i * Wl + j;
+                    const float ll = __ldg(q), lh = __ldg(q + S), hl = __ldg(q + 2 * S), hh = __ldg(q + 3 * S);
+                    const float pp = ll + lh, pm = ll - lh, qp = hl + hh, qm = hl - hh;
+                    a[2 * ci][2 * cj] = fmaf(0.5f, pp + qp, a[2 * ci][2 * cj]);
+                    a[2 * ci][2 * cj + 1] = fmaf(0.5f, pp - qp, a[2 * ci][2 * cj + 1]);
+                    a[2 * ci + 1][2 * cj] = fmaf(0.5f, pm + qm, a[2 * ci + 1][2 * cj]);
+                    a[2 * ci + 1][2 * cj + 1] = fmaf(0.5f, pm - qm, a[2 * ci + 1][2 * cj + 1]);
+                }
+            }
+    }
+    if (L >= 2) {
+        float deep = 0.f, scale = 0.25f;
+        for (int l = 3; l <= L; ++l) {
+            scale *= 0.5f;
+            const int Wl = lv.Wl[l - 1];
+            const size_t S = (size_t)lv.Hl[l - 1] * Wl;
+            const float *q = lv.z[l - 1] + p * 4 * S + (size_t)(Y0 >> l) * Wl + (X0 >> l);
+            deep += synth_term(__ldg(q), __ldg(q + S), __ldg(q + 2 * S), __ldg(q + 3 * S), (Y0 >> (l - 1)) & 1,
+                               (X0 >> (l - 1)) & 1, scale);
+        }
+        const int Wl = lv.Wl[1];
+        const size_t S = (size_t)lv.Hl[1] * Wl;
+        const float *q = lv.z[1] + p * 4 * S + (size_t)(Y0 >> 2) * Wl + (X0 >> 2);
+        const float ll = __ldg(q), lh = __ldg(q + S), hl = __ldg(q + 2 * S), hh = __ldg(q + 3 * S);
+        const float pp = ll + lh, pm = ll - lh, qp = hl + hh, qm = hl - hh;
+        float t2[2][2];
+        t2[0][0] = fmaf(0.25f, pp + qp, deep);
+        t2[0][1] = fmaf(0.25f, pp - qp, deep);
+        t2[1][0] = fmaf(0.25f, pm + qm, deep);
+        t2[1][1] = fmaf(0.25f, pm - qm, deep);
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) a[r][c] += t2[r >> 1][c >> 1];
+    }
+}
+
+// Store the block's rows that lie inside the image; whole aligned rows go out as one vector store.
+__device__ __forceinline__ void store4(float *p, const float *v) { *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+__device__ __forceinline__ void store4(__half *p, const float *v) {
+    const __half2 a = __floats2half2_rn(v[0], v[1]), b = __floats2half2_rn(v[2], v[3]);
+    uint2 q;
+    q.x = *reinterpret_cast<const unsigned *>(&a);
+    q.y = *reinterpret_cast<const unsigned *>(&b);
+    *reinterpret_cast<uint2 *>(p) = q;
+}
+__device__ __forceinline__ void store4(__nv_bfloat16 *p, const float *v) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    uint2 q;
+    q.x = *reinterpret_cast<const unsigned *>(&a);
+    q.y = *reinterpret_cast<const unsigned *>(&b);
+    *reinterpret_cast<uint2 *>(p) = q;
+}
+template <typename T>
+__device__ __forceinline__ void store_block(T *__restrict__ plane, int H, int W, int Y0, int X0, const float (&a)[4][4]) {
+    const bool vec = (W & 3) == 0 && X0 + 3 < W;  // base pointers are 16-byte aligned and the row pitch keeps it
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        if (Y0 + r >= H) break;
+        T *q = plane + (size_t)(Y0 + r) * W + X0;
+        if (vec) {
+            store4(q, a[r]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (X0 + c < W) stf(q + c, a[r][c]);
+        }
+    }
+}
+
 template <typename T, int K>
 __global__ void __launch_bounds__(NTHREADS)
 synth_fwd_kernel(const T *__restrict__ x, int H, int W, int C, int L, const float *__restrict__ w0,
                  const float *__restrict__ s0, const float *__restrict__ b0, LevelPtrs lv, T *__restrict__ out) {
-    constexpr int R = K / 2, SW = TW + 2 * R, SH = TH + 2 * R;
-    __shared__ float Xs[SH][SW + 1];
+    using S = SynthTile<K>;
+    __shared__ __align__(16) float Xs[S::XH][S::XP];
     const int p = blockIdx.x, c = p % C;
-    const int x0 = blockIdx.y * TW, y0 = blockIdx.z * TH;
-    const T *xp = x + (size_t)p * H * W;
-    for (int e = threadIdx.x; e < SH * SW; e += NTHREADS) {
-        int ly = e / SW, lx = e - ly * SW;
-        int yy = y0 + ly - R, xx = x0 + lx - R;
-        Xs[ly][lx] = (yy >= 0 && yy < H && xx >= 0 && xx < W) ? ldf(xp + (size_t)yy * W + xx) : 0.f;
-    }
-    float wr[K * K];
+    const int x0 = blockIdx.y * STW, y0 = blockIdx.z * STH;
+    stage_pixels<T, K>(x + (size_t)p * H * W, H, W, y0, x0, Xs);
+    // folded weights (Eq. 8) go through shared memory once, then live in registers
+    __shared__ float Ws[K * K + 1];
     const float sc = __ldg(s0 + c);
-#pragma unroll
-    for (int t = 0; t < K * K; ++t) wr[t] = sc * __ldg(w0 + (size_t)c * K * K + t);
-    const float bias = b0 ? sc * __ldg(b0 + c) : 0.f;
+    if (threadIdx.x < K * K) Ws[threadIdx.x] = sc * __ldg(w0 + (size_t)c * K * K + threadIdx.x);
+    if (threadIdx.x == K * K) Ws[K * K] = b0 ? sc * __ldg(b0 + c) : 0.f;
     __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int xx = x0 + lane;
+    float wr[K * K];
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const int ly = warp * 2 + r, yy = y0 + ly;
-        if (yy >= H || xx >= W) continue;
-        float acc = bias;
+    for (int t = 0; t < K * K; ++t) wr[t] = Ws[t];
+    const float bias = Ws[K * K];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int X0 = x0 + 4 * tx, Y0 = y0 + 4 * ty;
+    if (X0 >= W || Y0 >= H) return;
+    float acc[4][4];
 #pragma unroll
-        for (int u = 0; u < K; ++u)
+    for (int r = 0; r < 4; ++r)
 #pragma unroll
-            for (int v = 0; v < K; ++v) acc = fmaf(wr[u * K + v], Xs[ly + u][lane + v], acc);
-        float scale = 1.f;
-        for (int l = 1; l <= L; ++l) {
-            scale *= 0.5f;
-            const int Hl = lv.Hl[l - 1], Wl = lv.Wl[l - 1];
-            const size_t S = (size_t)Hl * Wl;
-            const float *zp = lv.z[l - 1] + (size_t)p * 4 * S + (size_t)(yy >> l) * Wl + (xx >> l);
-            acc += synth_term(__ldg(zp), __ldg(zp + S), __ldg(zp + 2 * S), __ldg(zp + 3 * S), (yy >> (l - 1)) & 1,
-                              (xx >> (l - 1)) & 1, scale);
-        }
-        stf(out + (size_t)p * H * W + (size_t)yy * W + xx, acc);
-    }
+        for (int cc = 0; cc < 4; ++cc) acc[r][cc] = bias;
+    block_conv<K, S::XP>(Xs, 4 * ty, 4 * tx, wr, acc);
+    block_synthesis(lv, L, (size_t)p, Y0, X0, acc);
+    store_block<T>(out + (size_t)p * H * W, H, W, Y0, X0, acc);
 }
 
 // Sum v over the 32 lanes; result valid in lane 0.
@@ -176,70 +384,72 @@ __device__ __forceinline__ float warp_sum(float v) {
 // grid (C * bsplit, tiles_x, tiles_y): block x = c * bsplit + part loops over batches
 // b = part, part + bsplit, ...  Partials: [C][nparts][4][K*K], nparts = tiles_x*tiles_y*bsplit.
 // ---------------------------------------------------------------------------------------------
+template <int K> constexpr size_t level_bwd_smem_bytes() {
+    return sizeof(float) * (2 * 4 * LevelTile<K>::H * LevelTile<K>::P + 8 * K * K + 4 * K * K);
+}
+
 template <typename Tin, int K>
 __global__ void __launch_bounds__(NTHREADS)
 level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, int Hp, int Wp, int Hl, int Wl, int B,
                  int C, int bsplit, const float *__restrict__ w, const float *__restrict__ s,
                  float *__restrict__ dY /* [P][4][Hl][Wl] */, float *__restrict__ Xl, float *__restrict__ Gl,
                  float *__restrict__ partials) {
-    constexpr int R = K / 2, KK = K * K;
-    __shared__ float Ys[4][TH + K - 1][TW + K];
-    __shared__ float Ds[4][TH + K - 1][TW + K];
-    __shared__ float red[8][KK];
+    using D = LevelTile<K>;
+    constexpr int KK = K * K;
+    extern __shared__ __align__(16) float lsm[];  // Ys[4][H][P], Ds[4][H][P], red[8][KK], Ws[4][KK]
+    float (*Ys)[D::H][D::P] = reinterpret_cast<float (*)[D::H][D::P]>(lsm);
+    float (*Ds)[D::H][D::P] = reinterpret_cast<float (*)[D::H][D::P]>(lsm + 4 * D::H * D::P);
+    float (*red)[KK] = reinterpret_cast<float (*)[KK]>(lsm + 8 * D::H * D::P);
+    float (*Ws)[KK] = reinterpret_cast<float (*)[KK]>(lsm + 8 * D::H * D::P + 8 * KK);
     const int c = blockIdx.x / bsplit, part = blockIdx.x - c * bsplit;
     const int j0 = blockIdx.y * TW, i0 = blockIdx.z * TH;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int sub = warp & 3, r0 = (warp >> 2) * ROWS_PER_THREAD;
+    const int sub = threadIdx.x >> 6, tx = threadIdx.x & 7, ty = (threadIdx.x >> 3) & 7;
+    const int I0 = i0 + 4 * ty, J0 = j0 + 4 * tx;
+    const bool live = I0 < Hl && J0 < Wl;
+    if (threadIdx.x < 4 * KK) {  // folded (Eq. 8) and rotated by 180 degrees
+        const int sb = threadIdx.x / KK, t = threadIdx.x % KK;
+        Ws[sb][t] = __ldg(s + c * 4 + sb) * __ldg(w + ((size_t)c * 4 + sb) * KK + (KK - 1 - t));
+    }
+    __syncthreads();
     float wf[KK], gw[KK];
-    const float sc = __ldg(s + c * 4 + sub);
 #pragma unroll
     for (int t = 0; t < KK; ++t) {
-        wf[t] = sc * __ldg(w + ((size_t)c * 4 + sub) * KK + (KK - 1 - t));  // folded and rotated by 180 degrees
+        wf[t] = Ws[sub][t];
         gw[t] = 0.f;
     }
-    const int j = j0 + lane;
     for (int b = part; b < B; b += bsplit) {
         const size_t p = (size_t)b * C + c;
         __syncthreads();
         stage_subbands<Tin, K>(Xprev + p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
         stage_subbands<Tin, K>(Gprev + p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ds);
         __syncthreads();
-        float acc[ROWS_PER_THREAD];
-        column_conv<K>(Ds[sub], r0, lane, wf, acc);
-        // weight gradient: this thread's 8 D values against the shifted Y window
-        float dcol[ROWS_PER_THREAD];
+        if (!live) continue;
+        // weight gradient: the block's 16 D values (zero outside the grid) against the shifted Y window
+        float d[4][4];
 #pragma unroll
-        for (int r = 0; r < ROWS_PER_THREAD; ++r) dcol[r] = Ds[sub][r0 + r + R][lane + R];
+        for (int r = 0; r < 4; ++r)
 #pragma unroll
-        for (int rr = 0; rr < ROWS_PER_THREAD + K - 1; ++rr) {
-            float in[K];
+            for (int cc = 0; cc < 4; ++cc) d[r][cc] = Ds[sub][4 * ty + D::R + r][4 * tx + D::R + cc];
+        block_wgrad<K, D::P>(Ys[sub], 4 * ty, 4 * tx, d, gw);
+        float acc[4][4];
 #pragma unroll
-            for (int v = 0; v < K; ++v) in[v] = Ys[sub][r0 + rr][lane + v];
+        for (int r = 0; r < 4; ++r)
 #pragma unroll
-            for (int u = 0; u < K; ++u) {
-                int r = rr - u;
-                if (r >= 0 && r < ROWS_PER_THREAD) {
+            for (int cc = 0; cc < 4; ++cc) acc[r][cc] = 0.f;
+        block_conv<K, D::P>(Ds[sub], 4 * ty, 4 * tx, wf, acc);
+        store_coeff_block(dY + (p * 4 + sub) * Hl * Wl, Hl, Wl, I0, J0, acc);
+        if (sub == 0 && Xl) {
+            float ll[4][4];
 #pragma unroll
-                    for (int v = 0; v < K; ++v) gw[u * K + v] = fmaf(dcol[r], in[v], gw[u * K + v]);
-                }
-            }
-        }
-        if (j < Wl) {
-            float *yp = dY + (p * 4 + sub) * Hl * Wl;
+            for (int r = 0; r < 4; ++r)
 #pragma unroll
-            for (int r = 0; r < ROWS_PER_THREAD; ++r) {
-                int i = i0 + r0 + r;
-                if (i < Hl) {
-                    yp[(size_t)i * Wl + j] = acc[r];
-                    if (sub == 0 && Xl) {
-                        Xl[(p * Hl + i) * Wl + j] = Ys[0][r0 + r + R][lane + R];
-                        Gl[(p * Hl + i) * Wl + j] = Ds[0][r0 + r + R][lane + R];
-                    }
-                }
-            }
+                for (int cc = 0; cc < 4; ++cc) ll[r][cc] = Ys[0][4 * ty + D::R + r][4 * tx + D::R + cc];
+            store_coeff_block(Xl + p * Hl * Wl, Hl, Wl, I0, J0, ll);
+            store_coeff_block(Gl + p * Hl * Wl, Hl, Wl, I0, J0, d);
         }
     }
-    // block reduction: lanes by shuffle, the two row halves of a subband through shared memory
+    // block reduction: lanes by shuffle, the two warps of a subband through shared memory
 #pragma unroll
     for (int t = 0; t < KK; ++t) {
         float v = warp_sum(gw[t]);
@@ -250,7 +460,7 @@ level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, i
     const int pidx = (blockIdx.z * gridDim.y + blockIdx.y) * bsplit + part;
     for (int e = threadIdx.x; e < 4 * KK; e += NTHREADS) {
         int sb = e / KK, t = e - sb * KK;
-        partials[(((size_t)c * nparts + pidx) * 4 + sb) * KK + t] = red[sb][t] + red[sb + 4][t];
+        partials[(((size_t)c * nparts + pidx) * 4 + sb) * KK + t] = red[2 * sb][t] + red[2 * sb + 1][t];
     }
 }
 
@@ -265,58 +475,50 @@ __global__ void __launch_bounds__(NTHREADS)
 synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W, int B, int C, int L, int bsplit,
                  const float *__restrict__ w0, const float *__restrict__ s0, LevelPtrs lv, T *__restrict__ dx,
                  float *__restrict__ partials) {
-    constexpr int R = K / 2, SW = TW + 2 * R, SH = TH + 2 * R, KK = K * K;
-    __shared__ float Xs[SH][SW + 1];
-    __shared__ float Gs[SH][SW + 1];
+    using S = SynthTile<K>;
+    constexpr int R = K / 2, KK = K * K;
+    __shared__ __align__(16) float Xs[S::XH][S::XP];
+    __shared__ __align__(16) float Gs[S::XH][S::XP];
     __shared__ float red[8][KK + 1];
     const int c = blockIdx.x / bsplit, part = blockIdx.x - c * bsplit;
-    const int x0 = blockIdx.y * TW, y0 = blockIdx.z * TH;
+    const int x0 = blockIdx.y * STW, y0 = blockIdx.z * STH;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int X0 = x0 + 4 * tx, Y0 = y0 + 4 * ty;
+    const bool live = X0 < W && Y0 < H;
     float wf[KK], gw[KK], gb = 0.f;
     const float sc = __ldg(s0 + c);
 #pragma unroll
     for (int t = 0; t < KK; ++t) {
-        wf[t] = sc * __ldg(w0 + (size_t)c * KK + (KK - 1 - t));
+        wf[t] = sc * __ldg(w0 + (size_t)c * KK + (KK - 1 - t));  // folded and rotated by 180 degrees
         gw[t] = 0.f;
     }
-    const int xx = x0 + lane;
     for (int b = part; b < B; b += bsplit) {
         const size_t p = (size_t)b * C + c;
-        const T *xp = x + p * H * W, *gp = g + p * H * W;
         __syncthreads();
-        for (int e = threadIdx.x; e < SH * SW; e += NTHREADS) {
-            int ly = e / SW, lx = e - ly * SW;
-            int yy = y0 + ly - R, xc = x0 + lx - R;
-            bool in = (yy >= 0 && yy < H && xc >= 0 && xc < W);
-            Xs[ly][lx] = in ? ldf(xp + (size_t)yy * W + xc) : 0.f;
-            Gs[ly][lx] = in ? ldf(gp + (size_t)yy * W + xc) : 0.f;
-        }
+        stage_pixels<T, K>(x + p * H * W, H, W, y0, x0, Xs);
+        stage_pixels<T, K>(g + p * H * W, H, W, y0, x0, Gs);
         __syncthreads();
+        if (!live) continue;
+        // weight gradient: the block's 16 upstream values (zero outside the image) against the shifted x window
+        float d[4][4];
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const int ly = warp * 2 + r, yy = y0 + ly;
-            if (yy >= H || xx >= W) continue;
-            float acc = 0.f;
-            const float gv = Gs[ly + R][lane + R];
-            gb += gv;
+        for (int r = 0; r < 4; ++r)
 #pragma unroll
-            for (int u = 0; u < K; ++u)
-#pragma unroll
-                for (int v = 0; v < K; ++v) {
-                    acc = fmaf(wf[u * K + v], Gs[ly + u][lane + v], acc);
-                    gw[u * K + v] = fmaf(gv, Xs[ly + u][lane + v], gw[u * K + v]);
-                }
-            float scale = 1.f;
-            for (int l = 1; l <= L; ++l) {
-                scale *= 0.5f;
-                const int Hl = lv.Hl[l - 1], Wl = lv.Wl[l - 1];
-                const size_t S = (size_t)Hl * Wl;
-                const float *zp = lv.z[l - 1] + p * 4 * S + (size_t)(yy >> l) * Wl + (xx >> l);
-                acc += synth_term(__ldg(zp), __ldg(zp + S), __ldg(zp + 2 * S), __ldg(zp + 3 * S), (yy >> (l - 1)) & 1,
-                                  (xx >> (l - 1)) & 1, scale);
+            for (int cc = 0; cc < 4; ++cc) {
+                d[r][cc] = Gs[4 * ty + R + r][4 * tx + R + cc];
+                gb += d[r][cc];
             }
-            stf(dx + p * H * W + (size_t)yy * W + xx, acc);
-        }
+        block_wgrad<K, S::XP>(Xs, 4 * ty, 4 * tx, d, gw);
+        // input gradient: rotated-kernel correlation of the upstream tile plus the Proposition 2 terms of dL/dY^l
+        float acc[4][4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) acc[r][cc] = 0.f;
+        block_conv<K, S::XP>(Gs, 4 * ty, 4 * tx, wf, acc);
+        block_synthesis(lv, L, p, Y0, X0, acc);
+        store_block<T>(dx + p * H * W, H, W, Y0, X0, acc);
     }
 #pragma unroll
     for (int t = 0; t < KK; ++t) {

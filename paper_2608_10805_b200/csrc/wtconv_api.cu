@@ -85,8 +85,8 @@ TiledPlan make_tiled_plan(const wtconv_desc *d) {
         p.gc_off[l - 1] = off;
         off = align_up(off + sizeof(float) * S * p.P);
     }
-    p.tx0 = cdiv(d->W, wt::tiled::TW);
-    p.ty0 = cdiv(d->H, wt::tiled::TH);
+    p.tx0 = cdiv(d->W, wt::tiled::STW);
+    p.ty0 = cdiv(d->H, wt::tiled::STH);
     p.bsplit0 = pick_bsplit(d->B, (long long)p.tx0 * p.ty0 * d->C);
     p.np0 = p.tx0 * p.ty0 * p.bsplit0;
     p.part0_off = off;
@@ -141,7 +141,7 @@ wtconv_status tiled_forward(const wtconv_desc *d, const T *x, const float *w0, c
         lv.Hl[l - 1] = Hl;
         lv.Wl[l - 1] = Wl;
     }
-    dim3 grid(pl.P, cdiv(d->W, TW), cdiv(d->H, TH));
+    dim3 grid(pl.P, cdiv(d->W, STW), cdiv(d->H, STH));
     synth_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, d->H, d->W, C, d->L, w0, s0, b0, lv, out);
     return launch_status();
 }
@@ -173,13 +173,19 @@ wtconv_status tiled_backward(const wtconv_desc *d, const T *x, const T *g, const
         float *part = (float *)(ws + pl.partl_off[l - 1]);
         dim3 grid(C * pl.bsplitl[l - 1], pl.txl[l - 1], pl.tyl[l - 1]);
         const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
-        if (l == 1)
-            level_bwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, g, Hp, Wp, Hl, Wl, d->B, C, pl.bsplitl[l - 1], wq, sq,
-                                                              dY, Xl, Gl, part);
-        else
-            level_bwd_kernel<float, K><<<grid, NTHREADS, 0, st>>>(
-                (const float *)(ws + pl.xc_off[l - 2]), (const float *)(ws + pl.gc_off[l - 2]), Hp, Wp, Hl, Wl, d->B, C,
-                pl.bsplitl[l - 1], wq, sq, dY, Xl, Gl, part);
+        constexpr size_t lsmem = level_bwd_smem_bytes<K>();  // above 48 KB for k = 7: opt in
+        if (l == 1) {
+            auto kern = level_bwd_kernel<T, K>;
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsmem) != cudaSuccess)
+                return WTCONV_ERR_CUDA;
+            kern<<<grid, NTHREADS, lsmem, st>>>(x, g, Hp, Wp, Hl, Wl, d->B, C, pl.bsplitl[l - 1], wq, sq, dY, Xl, Gl, part);
+        } else {
+            auto kern = level_bwd_kernel<float, K>;
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsmem) != cudaSuccess)
+                return WTCONV_ERR_CUDA;
+            kern<<<grid, NTHREADS, lsmem, st>>>((const float *)(ws + pl.xc_off[l - 2]), (const float *)(ws + pl.gc_off[l - 2]),
+                                                Hp, Wp, Hl, Wl, d->B, C, pl.bsplitl[l - 1], wq, sq, dY, Xl, Gl, part);
+        }
         lv.z[l - 1] = dY;
         lv.Hl[l - 1] = Hl;
         lv.Wl[l - 1] = Wl;
