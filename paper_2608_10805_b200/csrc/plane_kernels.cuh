@@ -19,6 +19,9 @@
 //    subband) class, so its 25 accumulators stay in registers across all images of a channel and are
 //    reduced once (block tree through shared memory, then fixed-order fp64 in the epilogue).
 #pragma once
+#include <cmath>
+#include <mutex>
+#include <vector>
 #include "common.cuh"
 #include "tiled_kernels.cuh"
 
@@ -1340,12 +1343,18 @@ inline bool plan_forward_th(int B, int C, int H, int W, int L, int elem_bytes, G
                 int nblocks = NUM_SMS * bps;
                 if (nblocks > units) nblocks = units;
                 // thread-slot use x resident warps (about 16 hide the latency-bound phases) x phase overlap
-                double occ = (double)bps * T / 384.0;
+                double occ = (double)bps * T / 512.0;
                 if (occ > 1.0) occ = 1.0;
                 const double overlap = bps >= 4 ? 1.0 : (bps == 3 ? 0.95 : (bps == 2 ? 0.8 : 0.55));
-                const double sc = teff * eff * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) * (rounds <= 2 ? 1.0 : 0.9) *
+                // more than 512 resident threads run the 80-register build, which spills with 8-row tiles and
+                // measured slower than four blocks of 128 threads on the smallest planes
+                const double regs = bps * T > 512 ? (th == 8 ? 0.75 : (T <= 128 ? 0.9 : 1.0)) : 1.0;
+                // small planes are bound by per-unit fixed costs: what counts is how many pixels are resident per SM
+                double inflight = (double)bps * npl * H * W / 8192.0;
+                inflight = inflight >= 1.0 ? 1.0 : pow(inflight, 0.3);
+                const double sc = teff * sqrt(eff) * (0.5 + 0.5 * occ) * overlap * (use_bulk ? 1.0 : 0.8) * (rounds <= 2 ? 1.0 : 0.9) *
                                   partition_eff(units, nblocks) * ((double)C / ((double)ngroups * npl)) *
-                                  (1.0 - 1e-4 * T / 32.0);
+                                  (1.0 - 1e-4 * T / 32.0) * regs * inflight;
                 if (sc > best.score + 1e-9) {
                     best = cg;
                     best.smem_floats = (int)smem_floats; best.ngroups = ngroups; best.units = units;
@@ -1499,7 +1508,7 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
 }
 
 // Each plan is searched for both tile heights; tune bit 22 forces 8 rows, bit 23 forces 4 rows.
-inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+inline bool search_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune) {
     best.score = -1.0;
     bool ok = false;
     if (!((tune >> 23) & 1)) ok |= plan_forward_th(B, C, H, W, L, elem_bytes, best, tune, 8);
@@ -1507,7 +1516,7 @@ inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom
     if (ok) deepen_prefetch(best);
     return ok;
 }
-inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+inline bool search_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune) {
     best.score = -1.0;
     bool ok = false;
     if (!((tune >> 23) & 1)) ok |= plan_wgrad_th(B, C, H, W, L, elem_bytes, best, tune, 8);
@@ -1515,7 +1524,7 @@ inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &
     if (ok) deepen_prefetch(best);
     return ok;
 }
-inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+inline bool search_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune) {
     if ((tune >> 21) & 1) return false;  // bit 21: never fuse
     best.score = -1.0;
     bool ok = false;
@@ -1523,6 +1532,57 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
     if (!((tune >> 22) & 1)) ok |= plan_bwd_fused_th(B, C, H, W, L, elem_bytes, best, tune, 4);
     if (ok) deepen_prefetch(best);
     return ok;
+}
+
+// The searches above walk a few thousand candidates (tens of microseconds of host time), more than a small
+// layer's kernels take on the GPU, so every entry point looks its plan up in a small process-wide cache first.
+struct PlanKey {
+    int kind, B, C, H, W, L, elem_bytes;
+    unsigned tune;
+    bool operator==(const PlanKey &o) const {
+        return kind == o.kind && B == o.B && C == o.C && H == o.H && W == o.W && L == o.L && elem_bytes == o.elem_bytes &&
+               tune == o.tune;
+    }
+};
+struct PlanEntry {
+    PlanKey key;
+    bool ok;
+    Geom g;
+};
+inline bool cached_plan(int kind, int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune) {
+    static std::mutex mu;
+    static std::vector<PlanEntry> cache;
+    const PlanKey key = {kind, B, C, H, W, L, elem_bytes, tune};
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        for (const PlanEntry &e : cache)
+            if (e.key == key) {
+                if (e.ok) best = e.g;
+                return e.ok;
+            }
+    }
+    PlanEntry e;
+    e.key = key;
+    e.g = Geom{};
+    e.ok = kind == 0   ? search_forward(B, C, H, W, L, elem_bytes, e.g, tune)
+           : kind == 1 ? search_wgrad(B, C, H, W, L, elem_bytes, e.g, tune)
+                       : search_bwd_fused(B, C, H, W, L, elem_bytes, e.g, tune);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (cache.size() >= 256) cache.clear();  // bounded: a process cycling through more shapes just searches again
+        cache.push_back(e);
+    }
+    if (e.ok) best = e.g;
+    return e.ok;
+}
+inline bool plan_forward(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    return cached_plan(0, B, C, H, W, L, elem_bytes, best, tune);
+}
+inline bool plan_wgrad(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    return cached_plan(1, B, C, H, W, L, elem_bytes, best, tune);
+}
+inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Geom &best, unsigned tune = 0) {
+    return cached_plan(2, B, C, H, W, L, elem_bytes, best, tune);
 }
 
 inline int dtype_bytes(int dtype) { return dtype == 0 ? 4 : 2; }
