@@ -1171,7 +1171,13 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
             for (int t = 0; t < KK; ++t) scr[tid * (KK + 2) + t] = accw[t];
             scr[tid * (KK + 2) + KK] = gsum;
-            scr[tid * (KK + 2) + KK + 1] = __int_as_float(item.meta < 0 ? item.slot * 64 + cls : -1);
+            const int mytag = item.meta < 0 ? item.slot * 64 + cls : -1;
+            scr[tid * (KK + 2) + KK + 1] = __int_as_float(mytag);
+            __syncthreads();
+            // the threads of one (plane, class) are neighbours in the item list: note where each run starts
+            int *run_start = reinterpret_cast<int *>(scr + nthr * (KK + 2));
+            if (mytag >= 0 && (tid == 0 || __float_as_int(scr[(tid - 1) * (KK + 2) + KK + 1]) != mytag))
+                run_start[item.slot * ncls + cls] = tid;
             __syncthreads();
             const int slotp = blockIdx.x - block_of_unit((long long)cg * g.B, gridDim.x, g.units);
             for (int e = tid; e < nvalid * ncls * (KK + 1); e += nthr) {
@@ -1179,8 +1185,8 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 if (c2 > 0 && t == KK) continue;
                 const int tag = slot * 64 + c2, ch = c + slot;
                 float sacc = 0.f;
-                for (int th = 0; th < nthr; ++th)
-                    if (__float_as_int(scr[th * (KK + 2) + KK + 1]) == tag) sacc += scr[th * (KK + 2) + t];
+                for (int th = run_start[sc]; th < nthr && __float_as_int(scr[th * (KK + 2) + KK + 1]) == tag; ++th)
+                    sacc += scr[th * (KK + 2) + t];
                 if (c2 == 0) {
                     part0[((size_t)ch * g.np + slotp) * (KK + 1) + t] = sacc;
                 } else {
@@ -1189,7 +1195,8 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 }
             }
             __syncthreads();
-            for (int i = tid; i < g.wtab_off; i += nthr) sm[i] = 0.f;  // restore the zero halos of the arrays
+            for (int i = tid; i < g.wtab_off / 4; i += nthr)  // restore the zero halos of the arrays
+                reinterpret_cast<float4 *>(sm)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int t = 0; t < KK; ++t) accw[t] = 0.f;
             gsum = 0.f;
@@ -1460,7 +1467,7 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
         const int wtab = npl * (1 + 4 * L) * WT_STRIDE;
         const int T = (npl * M + 31) & ~31;
         long long arrays = (long long)npl * slot;
-        const long long scratch = (long long)T * (KK + 2);
+        const long long scratch = (long long)T * (KK + 2) + (long long)npl * (1 + 4 * L);  // flush scratch: sums, tags, run starts
         if (scratch > arrays) arrays = scratch;
         const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 20) & 1);
         bool any = false;
