@@ -389,7 +389,7 @@ template <int K> constexpr size_t level_bwd_smem_bytes() {
 }
 
 template <typename Tin, int K>
-__global__ void __launch_bounds__(NTHREADS)
+__global__ void __launch_bounds__(NTHREADS, K <= 5 ? 3 : 1)
 level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, int Hp, int Wp, int Hl, int Wl, int B,
                  int C, int bsplit, const float *__restrict__ w, const float *__restrict__ s,
                  float *__restrict__ dY /* [P][4][Hl][Wl] */, float *__restrict__ Xl, float *__restrict__ Gl,
@@ -471,7 +471,7 @@ level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, i
 // grid (C * bsplit, tiles_x, tiles_y).  Partials: [C][nparts][K*K + 1].
 // ---------------------------------------------------------------------------------------------
 template <typename T, int K>
-__global__ void __launch_bounds__(NTHREADS)
+__global__ void __launch_bounds__(NTHREADS, K <= 5 ? 3 : 1)
 synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W, int B, int C, int L, int bsplit,
                  const float *__restrict__ w0, const float *__restrict__ s0, LevelPtrs lv, T *__restrict__ dx,
                  float *__restrict__ partials) {
