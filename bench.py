@@ -32,8 +32,8 @@ FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FP32 lanes x 2 FL
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (bytes; keyed by workload and kernel).  None where no capture exists.
 NCU_DRAM_TRAFFIC = {
-    ("stage1_f32", "plane_bwd_kernel"): 154784768 + 49147648,
-    ("stage1_f32", "plane_fwd_kernel"): 77334528 + 32297984,
+    ("stage1_f32", "plane_bwd_kernel"): 154790144 + 48572416,
+    ("stage1_f32", "plane_fwd_kernel"): 77372416 + 32101632,
 }
 
 
@@ -309,7 +309,7 @@ def main():
             "alu_floor_ms": fl_step / (FP32_ALU_PEAK_TFLOPS * 1e12) * 1e3,
             "hbm_floor_ms": hbm_step / (peaks["hbm_gbs"] * 1e9) * 1e3},
         "paper_io_model": {"q_fused_fwd_N": io_model.q_fused(wl.L), "q_ref_fwd_N": io_model.q_ref(wl.L),
-                           "ours_fwd_N": 2.0, "ours_bwd_N": 4.0},
+                           "ours_fwd_N": 2.0, "ours_bwd_N": 3.0 if nb == 2 else 4.0},
     }
     if world == 1 and not args.no_cpu_baseline:
         from oracle import wtconv_oracle as O
