@@ -104,6 +104,31 @@ def test_scratch_memory_accounting(lib):
     assert abs(fb - 4 * P * coeffs) <= 4096 * (wl.L + 2), (fb, 4 * P * coeffs)
 
 
+def test_host_planning_over_a_shape_sweep(lib):
+    """The host-side planners (pure integer code) give a plan, a launch count and a workspace size for every
+    shape in a sweep that crosses the plane / tiled boundary, odd sizes, L = 0 and grids that shrink to 1 x 1."""
+    seen = set()
+    for H, W in [(1, 1), (1, 19), (7, 7), (9, 12), (13, 9), (14, 14), (28, 28), (29, 29), (56, 56), (57, 33), (64, 64),
+                 (70, 66), (71, 71), (96, 40), (128, 128), (225, 225)]:
+        for L in (0, 1, 2, 3, 5, 8):
+            for dt in ("f32", "bf16"):
+                for B, C in ((1, 1), (2, 3), (64, 96), (128, 768)):
+                    d = wt.make_desc(B, C, H, W, 5, L, dt)
+                    name = wt.wtconv_plan_name(d)
+                    assert name in ("plane", "tiled"), (H, W, L, dt, B, C, name)
+                    seen.add(name)
+                    nf, nb = wt.wtconv_launch_count(d)
+                    if name == "plane":
+                        assert nf == 1 and nb in (2, 3)
+                    else:
+                        assert nf == L + 1 and nb == L + 2
+                    fb, bb = wt.wtconv_workspace_bytes(d)
+                    assert fb >= (256 if name == "plane" else 0) and bb >= fb and bb > 0 and fb % 256 == 0 and bb % 256 == 0, (H, W, L, dt, B, C, fb, bb)
+                    for lvl in range(L + 1):
+                        assert wt.wtconv_level_shape(d, lvl) == (-(-H // (1 << lvl)), -(-W // (1 << lvl)))
+    assert seen == {"plane", "tiled"}
+
+
 def test_binding_refuses_to_run_without_the_library(monkeypatch):
     monkeypatch.setattr(wt, "_lib", None)
     monkeypatch.setattr(wt, "LIB_PATH", "/nonexistent/libwtconv_b200.so")
