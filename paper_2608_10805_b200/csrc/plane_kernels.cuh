@@ -496,6 +496,16 @@ __device__ __forceinline__ void zero_fill(float *sm, const Geom &g) {
     for (int i = g.out_off / 4 + threadIdx.x; i < g.bar_off / 4; i += blockDim.x) v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
+// Without room for a raw prefetch buffer the next unit is at least pulled into L2: every thread touches some of
+// the unit's 128-byte lines (prefetch only; no registers or shared memory are tied up).
+template <typename T>
+__device__ __forceinline__ void prefetch_unit_l2(const Geom &g, const T *__restrict__ src, int c0, int b) {
+    const char *base = reinterpret_cast<const char *>(src + ((size_t)b * g.C + c0) * g.H * g.W);
+    const int bytes = g.NPL * g.plane_bytes;
+    for (int o = threadIdx.x * 128; o < bytes; o += blockDim.x * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + o));
+}
+
 // Issue the bulk copy of one unit's planes into the raw buffer (one thread); a second tensor (grad_out) goes
 // right behind the first on the same barrier.
 template <typename T>
@@ -798,6 +808,9 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                                      (u + g.nstage) - cgn * g.B);
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
+        } else if (u + 1 < u_end) {  // no room for a raw buffer: at least warm the next unit in L2
+            const int cgn = fdiv(u + 1, g.d_B);
+            if (cgn * g.NPL + g.NPL <= g.C) prefetch_unit_l2<T>(g, x, cgn * g.NPL, (u + 1) - cgn * g.B);
         }
         WT_TICK(3);
         for (int l = lnext; l <= L; ++l) {
@@ -917,6 +930,10 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
                                      (u + g.nstage) - cgn * g.B);
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
+        } else if (u + 1 < u_end) {
+            const int cn = fdiv(u + 1, g.d_B), bn = (u + 1) - cn * g.B;
+            prefetch_unit_l2<T>(g, x, cn, bn);
+            prefetch_unit_l2<T>(g, go, cn, bn);
         }
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
@@ -1087,6 +1104,13 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                                      (u + g.nstage) - cgn * g.B);
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
+        }
+        if (BULK != 2 && u + 1 < u_end) {  // what does not come by bulk copy is warmed in L2 behind this unit's math
+            const int cgn = fdiv(u + 1, g.d_B), bn = (u + 1) - cgn * g.B;
+            if (cgn * g.NPL + g.NPL <= g.C) {
+                if (BULK == 0) prefetch_unit_l2<T>(g, x, cgn * g.NPL, bn);
+                prefetch_unit_l2<T>(g, go, cgn * g.NPL, bn);
+            }
         }
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
