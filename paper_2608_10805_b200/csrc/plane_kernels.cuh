@@ -1045,9 +1045,18 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     bool has_base = false;
     const ItemD item = decode_item(g, tid, nlevel_items, nitems, bslot, tyy, txx, has_base);
     const int cls = (item.meta >> 24) & 0x3f;
-    const bool hoist_patch = g.vec && L >= 2 && g.NPL * g.npatch4 <= 2 * nthr;
-    const PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? tid : 0x3fffffff);
-    const PatchD patch1 = decode_patch(g, g.offA, hoist_patch ? tid + nthr : 0x3fffffff);
+    // No barrier separates a unit's synthesis (which reads only Z and registers) from the next unit's staging.
+    // With the planes already in shared memory (BULK == 2) the staging is left to the whole warps that hold
+    // level tiles only, two patches each if need be, while the base-tile threads finish the synthesis.  With
+    // staging from global memory every thread takes part: two patches per thread would make the exposed
+    // load-to-store chain twice as long (measured slower at 56 x 56 fp32).
+    int nstagers = (nlevel_items / 32) * 32;
+    if (nstagers > nthr) nstagers = nthr;
+    if (BULK != 2 || nstagers * 4 < nthr || g.NPL * g.npatch4 > 2 * nstagers) nstagers = nthr;
+    const int srank = tid < nstagers ? tid : 0x3fffffff;
+    const bool hoist_patch = g.vec && L >= 2 && g.NPL * g.npatch4 <= 2 * nstagers;
+    const PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
+    const PatchD patch1 = decode_patch(g, g.offA, hoist_patch && srank < nstagers ? srank + nstagers : 0x3fffffff);
     const int dA0 = g.offG[0] - g.offA[0], dA1 = L >= 1 ? g.offG[1] - g.offA[1] : 0, dA2 = L >= 2 ? g.offG[2] - g.offA[2] : 0;
     float accw[KK], gsum = 0.f;
 #pragma unroll
@@ -1224,8 +1233,11 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
             for (int t = 0; t < KK; ++t) accw[t] = 0.f;
             gsum = 0.f;
+            __syncthreads();  // the arrays are zeroed again before anybody stages into them
         }
-        __syncthreads();  // arrays and Z are free again for the next unit's staging
+        // No barrier here: the next unit's staging overwrites x / Y / D (last read before the barrier that
+        // follows the tile phase) while the base-tile threads may still run this unit's synthesis, which
+        // reads only Z (next written after the staging barriers) and registers.
     }
     if (BULK && g.bulk_out && tid == 0) bulk_store_wait_read();
 }
