@@ -165,7 +165,10 @@ wtconv_status wtconv_backward_static(const wtconv_desc *desc, const void *x, con
  * gradients back, all asynchronously on `stream` (the host buffers should be pinned for the
  * copies to overlap; they must stay valid until the stream reaches this point).
  * Every h_* pointer is a HOST pointer with the layouts above; `workspace` is DEVICE scratch of
- * at least wtconv_step_host_workspace_bytes.  h_b0 / h_grad_b0 may both be NULL. */
+ * at least wtconv_step_host_workspace_bytes.  h_b0 / h_grad_b0 may both be NULL.
+ * The forward result is copied back on a library-internal stream (one per device, created on the first
+ * call) while grad_out is still being uploaded; `stream` waits for that copy, so everything is complete
+ * when `stream` reaches this point.  The first call on a device must not happen inside a stream capture. */
 wtconv_status wtconv_step_host_workspace_bytes(const wtconv_desc *desc, size_t *bytes);
 wtconv_status wtconv_step_host(const wtconv_desc *desc, const void *h_x, const void *h_grad_out,
                                const float *h_w0, const float *h_s0, const float *h_b0,

@@ -296,6 +296,19 @@ wtconv_status static_scratch_for_current_device(void **out) {
     return WTCONV_OK;
 }
 
+// Internal copy stream of wtconv_step_host, one per device, created on first use and kept for the process.
+std::mutex g_side_mutex;
+cudaStream_t g_side_stream[MAX_DEVICES] = {};
+wtconv_status side_stream_for_current_device(cudaStream_t *out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return WTCONV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    if (!g_side_stream[dev] && cudaStreamCreateWithFlags(&g_side_stream[dev], cudaStreamNonBlocking) != cudaSuccess)
+        return WTCONV_ERR_CUDA;
+    *out = g_side_stream[dev];
+    return WTCONV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -444,8 +457,22 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     auto d2h = [&](void *dst, const void *src, size_t n) {
         if (n) ok = ok && cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, cs) == cudaSuccess;
     };
+    // The forward needs only x: its result travels back on an internal stream while grad_out is still on its
+    // way up (the link is full duplex), and `stream` waits for that copy before it reaches the end of the step.
+    cudaStream_t side = nullptr;
+    if ((st = side_stream_for_current_device(&side)) != WTCONV_OK) return st;
+    cudaEvent_t fwd_done = nullptr, out_home = nullptr;
+    if (cudaEventCreateWithFlags(&fwd_done, cudaEventDisableTiming) != cudaSuccess) return WTCONV_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&out_home, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventDestroy(fwd_done);
+        return WTCONV_ERR_CUDA;
+    }
+    // the events are released as soon as the work recorded so far has passed them
+    struct EventGuard {
+        cudaEvent_t a, b;
+        ~EventGuard() { cudaEventDestroy(a); cudaEventDestroy(b); }
+    } guard = {fwd_done, out_home};
     h2d(dx_, h_x, act_raw);
-    h2d(dg, h_g, act_raw);
     h2d(w0, h_w0, ps.w0);
     h2d(s0, h_s0, ps.s0);
     if (h_b0) h2d(b0, h_b0, ps.s0);
@@ -455,16 +482,25 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     const float *b0p = h_b0 ? b0 : nullptr;
     st = wtconv_forward(d, dx_, w0, s0, b0p, wl, sl, dout, p, rest, stream);
     if (st != WTCONV_OK) return st;
+    ok = ok && cudaEventRecord(fwd_done, cs) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(side, fwd_done, 0) == cudaSuccess;
+    if (ok) ok = cudaMemcpyAsync(h_out, dout, act_raw, cudaMemcpyDeviceToHost, side) == cudaSuccess;
+    ok = ok && cudaEventRecord(out_home, side) == cudaSuccess;
+    h2d(dg, h_g, act_raw);
+    if (!ok) return WTCONV_ERR_CUDA;
     st = wtconv_backward(d, dx_, dg, w0, s0, b0p, wl, sl, dgx, gw0, gs0, h_b0 ? gb0 : nullptr, gwl, gsl, p, rest,
                          stream);
-    if (st != WTCONV_OK) return st;
-    d2h(h_out, dout, act_raw);
+    if (st != WTCONV_OK) {
+        cudaStreamWaitEvent(cs, out_home, 0);
+        return st;
+    }
     d2h(h_gx, dgx, act_raw);
     d2h(h_gw0, gw0, ps.w0);
     d2h(h_gs0, gs0, ps.s0);
     if (h_b0) d2h(h_gb0, gb0, ps.s0);
     d2h(h_gwl, gwl, ps.wl);
     d2h(h_gsl, gsl, ps.sl);
+    ok = ok && cudaStreamWaitEvent(cs, out_home, 0) == cudaSuccess;  // join: the step ends when `out` is home too
     return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
 }
 
