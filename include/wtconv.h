@@ -65,7 +65,7 @@ typedef enum {
     WTCONV_ERR_ALIAS = 8,       /* an output overlaps an input */
     WTCONV_ERR_ARCH = 9,        /* the current device is not compute capability 10.x */
     WTCONV_ERR_CUDA = 10,       /* a CUDA runtime call or launch failed */
-    WTCONV_ERR_TIMEOUT = 11     /* reserved: a bounded device-side wait ran out */
+    WTCONV_ERR_TIMEOUT = 11     /* a bounded device-side wait ran out (see wtconv_read_status) */
 } wtconv_status;
 
 #define WTCONV_MAX_LEVELS 8
@@ -132,6 +132,16 @@ wtconv_status wtconv_backward(const wtconv_desc *desc, const void *x, const void
                               void *grad_x, float *grad_w0, float *grad_s0, float *grad_b0,
                               float *grad_wl, float *grad_sl,
                               void *workspace, size_t workspace_bytes, void *stream);
+
+/* Device-side status of the last call that used `workspace` (device pointer) with this descriptor: enqueues on
+ * `stream` a copy of the workspace's status word into *h_flag (a HOST int32, pinned if the copy is to be
+ * asynchronous).  Once the stream has reached this point, 0 means every bounded wait inside the kernels
+ * completed (the paper's kernels wait for nothing; ours wait only for their own bulk copies); non-zero means a
+ * wait ran out and the outputs of that call are not valid (report it as WTCONV_ERR_TIMEOUT).  For descriptors
+ * served by the tiled kernels, which wait for nothing, *h_flag is set to 0 at once.  The library itself never
+ * synchronises, so it cannot return that code from wtconv_forward / wtconv_backward.
+ * Errors: NULL, the descriptor's own errors, ALIGNMENT (workspace), CUDA. */
+wtconv_status wtconv_read_status(const wtconv_desc *desc, const void *workspace, int32_t *h_flag, void *stream);
 
 /* Backward pass for callers that cannot hand over a workspace.  (The paper has no counterpart: it never
  * discusses where its kernels' scratch comes from.)

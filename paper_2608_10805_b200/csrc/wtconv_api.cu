@@ -504,6 +504,21 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
 }
 
+wtconv_status wtconv_read_status(const wtconv_desc *d, const void *workspace, int32_t *h_flag, void *stream) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (!workspace || !h_flag) return WTCONV_ERR_NULL;
+    if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
+    if (!use_plane_path(d)) {  // the tiled kernels wait for nothing and keep no status word
+        *h_flag = 0;
+        return WTCONV_OK;
+    }
+    // the status word is the first word of every workspace the plane kernels use
+    return cudaMemcpyAsync(h_flag, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream) == cudaSuccess
+               ? WTCONV_OK
+               : WTCONV_ERR_CUDA;
+}
+
 wtconv_status wtconv_backward_static(const wtconv_desc *d, const void *x, const void *grad_out, const float *w0,
                                      const float *s0, const float *b0, const float *wl, const float *sl, void *grad_x,
                                      float *grad_w0, float *grad_s0, float *grad_b0, float *grad_wl, float *grad_sl,

@@ -19,7 +19,7 @@ _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_NAMES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
 
 EXPORTS = ["wtconv_status_string", "wtconv_level_shape", "wtconv_workspace_bytes", "wtconv_plan_name",
-           "wtconv_launch_count", "wtconv_forward", "wtconv_backward", "wtconv_backward_static",
+           "wtconv_launch_count", "wtconv_forward", "wtconv_backward", "wtconv_read_status", "wtconv_backward_static",
            "wtconv_step_host_workspace_bytes", "wtconv_step_host"]
 
 
@@ -56,6 +56,7 @@ def lib():
         L.wtconv_forward.argtypes = [dp] + [vp] * 7 + [vp, sz, vp]
         L.wtconv_backward.argtypes = [dp] + [vp] * 13 + [vp, sz, vp]
         L.wtconv_backward_static.argtypes = [dp] + [vp] * 13 + [vp]
+        L.wtconv_read_status.argtypes = [dp, vp, vp, vp]
         L.wtconv_step_host_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz)]
         L.wtconv_step_host.argtypes = [dp] + [vp] * 14 + [vp, sz, vp]
         _lib = L
@@ -126,6 +127,14 @@ def wtconv_backward(desc, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad
     _check(lib().wtconv_backward(ctypes.byref(desc), _ptr(x), _ptr(grad_out), _ptr(w0), _ptr(s0), _ptr(b0), _ptr(wl),
                                  _ptr(sl), _ptr(grad_x), _ptr(grad_w0), _ptr(grad_s0), _ptr(grad_b0), _ptr(grad_wl),
                                  _ptr(grad_sl), _ptr(workspace), workspace.numel(), _stream(stream)))
+
+
+def wtconv_read_status(desc, workspace, h_flag, stream=None):
+    """Enqueue a copy of the workspace's device status word into the host int32 tensor `h_flag` (pin it)."""
+    _need_cuda(workspace)
+    if h_flag.is_cuda or h_flag.dtype != torch.int32 or h_flag.numel() < 1:
+        raise ValueError("h_flag must be a host int32 tensor")
+    _check(lib().wtconv_read_status(ctypes.byref(desc), _ptr(workspace), _ptr(h_flag), _stream(stream)))
 
 
 STATIC_SCRATCH_BYTES = 8 << 20

@@ -68,3 +68,14 @@ def test_overlapping_calls_from_several_threads_match_serial_results():
         assert torch.equal(out, sout)  # same kernels on the same data: bit-identical
         for k, v in sgr.items():
             assert torch.equal(gr[k], v), k
+
+
+@pytest.mark.parametrize("wl", CASES, ids=lambda w: w.name)
+def test_status_word_reads_zero_after_a_normal_step(wl):
+    desc, t = _setup(wl)
+    s = torch.cuda.Stream()
+    out, gr, ws = _run(desc, t, s)
+    flag = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    wt.wtconv_read_status(desc, ws, flag, s)
+    s.synchronize()
+    assert int(flag[0]) == 0 and bool(torch.isfinite(out.float()).all())
