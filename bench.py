@@ -32,8 +32,8 @@ FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FP32 lanes x 2 FL
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (bytes; keyed by workload and kernel).  None where no capture exists.
 NCU_DRAM_TRAFFIC = {
-    ("stage1_f32", "plane_bwd_kernel"): 154790144 + 48572416,
-    ("stage1_f32", "plane_fwd_kernel"): 77372416 + 32101632,
+    ("stage1_f32", "plane_bwd_kernel"): 154664704 + 48539904,
+    ("stage1_f32", "plane_fwd_kernel"): 77319680 + 32544768,
 }
 
 
