@@ -1,23 +1,34 @@
 // Whole-plane WTConv kernels for sm_100a (k = 5): every (b, c) plane's entire decomposition lives
-// in shared memory, so the only HBM traffic is the compulsory one (read x, write out).
+// in shared memory, so the only HBM traffic is the compulsory one (read x, write out; in the backward
+// read x and grad_out, write grad_x).
 //
 // Design
-//  * A block works on units of NPL planes of one channel (images b0..b0+NPL-1).  A plane's footprint
-//    (x with a zero halo, the four Haar subbands of every level with halos, the conv outputs Z^l) is
-//    about 58 KB for 56x56, so three to four blocks are resident per SM: while one block is in a
+//  * A block is persistent and walks a contiguous range of units.  A unit is NPL consecutive channels of
+//    one image (contiguous in NCHW, so one aligned bulk copy fetches it); units are ordered channel-group
+//    major, so a block keeps its folded weight table (Eq. 8) over all images of a group.  A plane's
+//    footprint (x with a zero halo, the four Haar subbands of every level with halos, the conv outputs
+//    Z^l) is about 58 KB for 56x56, so three blocks are resident per SM: while one block is in a
 //    latency-bound phase (staging, synthesis, stores) the others keep the FP32 pipe busy.
-//  * Per unit: stage x into the haloed array and run the Haar butterfly of Eq. 5 on chip (Sec. 4.1),
-//    level by level from the raw LL band; then every thread convolves 4-column x 8-row register tiles
-//    straight out of shared memory (two aligned 16-byte loads per window row, lanes 16 bytes apart: no
-//    bank conflicts) with weights that already carry the scale (Eq. 8).  Level tiles and base tiles are
-//    one item list and one code path; a thread keeps its base tile in registers across one barrier and
-//    then adds the bit-indexed closed-form synthesis of Proposition 2 (Sec. 4.2) before the only store.
-//  * Backward = two kernels.  grad_x is the same kernel run on grad_out with the kernels rotated by 180
-//    degrees (Sec. 2.2: the adjoint of analysis is synthesis and vice versa, so the adjoint of the whole
-//    operator has the operator's own structure).  The weight-gradient kernel stages the decompositions
-//    of x and grad_out and correlates them tile by tile; each thread only ever works on one (level,
-//    subband) class, so its 25 accumulators stay in registers across all images of a channel and are
-//    reduced once (block tree through shared memory, then fixed-order fp64 in the epilogue).
+//  * Units arrive through a ring of raw buffers filled by cp.async.bulk and watched by mbarriers (bounded
+//    waits that raise a status word instead of spinning for ever); where no ring fits, the next unit is
+//    warmed in L2.  Per unit: stage x into the haloed array and run the Haar butterfly of Eq. 5 on chip
+//    (Sec. 4.1), levels 1 and 2 in the same pass, deeper levels from the raw LL band; then every thread
+//    convolves 4-column x TH-row register tiles (TH = 4 or 8, chosen per plan) straight out of shared
+//    memory (two aligned 16-byte loads per window row) with weights that already carry the scale.  Level
+//    tiles and base tiles are one item list and one rolled copy of the tile code; a thread keeps its base
+//    tile in registers across one barrier and then adds the bit-indexed closed-form synthesis of
+//    Proposition 2 (Sec. 4.2) before the only store.
+//  * Backward.  grad_x is the forward dataflow run on grad_out with the kernels rotated by 180 degrees
+//    (Sec. 2.2: the adjoint of analysis is synthesis and vice versa, so the adjoint of the whole operator
+//    has the operator's own structure).  The fused kernel stages the decompositions of x and grad_out
+//    once; every thread owns one tile, first correlates it into the 25 weight-gradient accumulators of
+//    its (level, subband) class - kept in registers across all images of a channel and reduced once by a
+//    block tree through shared memory, then in fixed-order fp64 in the epilogue - and then runs the
+//    rotated-kernel convolution, synthesis and store on the same window.  Shapes whose tiles do not fit
+//    one pass of 256 threads take the split pair instead: a weight-gradient kernel with class-major
+//    thread allocation plus the FLIP instantiation of the forward kernel.
+//  * Host side: plans (threads, blocks per SM, planes per unit, tile height, ring depth) come from a
+//    search over a small cost model and are cached per shape.
 #pragma once
 #include <cmath>
 #include <mutex>
