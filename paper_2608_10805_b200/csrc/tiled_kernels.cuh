@@ -31,6 +31,21 @@ template <int K, int TWc, int THc> struct TileDims {
 };
 template <int K> using LevelTile = TileDims<K, TW, TH>;
 
+// Four consecutive activations as floats (16-byte / 8-byte aligned vector load).
+__device__ __forceinline__ float4 load_vec4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ float4 load_vec4(const __half *p) {
+    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ float4 load_vec4(const __nv_bfloat16 *p) {
+    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+}
+
 // Two horizontally adjacent activations as floats (the pair starts at an even column of an even-length row, so
 // it is aligned to its own size).
 __device__ __forceinline__ float2 load_pair(const float *p) { return __ldg(reinterpret_cast<const float2 *>(p)); }
@@ -50,6 +65,28 @@ template <typename Tin, int K>
 __device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int Hp, int Wp, int Hl, int Wl, int i0,
                                                int j0, float (*Ys)[LevelTile<K>::H][LevelTile<K>::P] /* [4] */) {
     using D = LevelTile<K>;
+    if ((D::R & 1) == 0 && (Wp & 3) == 0) {
+        // two coefficients per step from one 4-pixel vector load per row: with an even halo and rows that are
+        // multiples of four pixels a pair (j even) is aligned and lies wholly inside or wholly outside the grid
+        for (int e = threadIdx.x; e < D::H * (D::P / 2); e += NTHREADS) {
+            const int li = e / (D::P / 2), lj = 2 * (e - li * (D::P / 2));
+            const int i = i0 + li - D::R, j = j0 + lj - D::R;
+            Haar4 h0 = {0.f, 0.f, 0.f, 0.f}, h1 = {0.f, 0.f, 0.f, 0.f};
+            if (lj < D::W && i >= 0 && i < Hl && j >= 0 && j < Wl) {
+                const Tin *q = xp + (size_t)(2 * i) * Wp + 2 * j;
+                const float4 t = load_vec4(q);
+                float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (2 * i + 1 < Hp) u = load_vec4(q + Wp);
+                h0 = haar_butterfly(t.x, t.y, u.x, u.y);
+                h1 = haar_butterfly(t.z, t.w, u.z, u.w);
+            }
+            *reinterpret_cast<float2 *>(&Ys[0][li][lj]) = make_float2(h0.ll, h1.ll);
+            *reinterpret_cast<float2 *>(&Ys[1][li][lj]) = make_float2(h0.lh, h1.lh);
+            *reinterpret_cast<float2 *>(&Ys[2][li][lj]) = make_float2(h0.hl, h1.hl);
+            *reinterpret_cast<float2 *>(&Ys[3][li][lj]) = make_float2(h0.hh, h1.hh);
+        }
+        return;
+    }
     const bool even = (Wp & 1) == 0;
     for (int e = threadIdx.x; e < D::H * D::P; e += NTHREADS) {
         const int li = e / D::P, lj = e - li * D::P;
@@ -205,21 +242,6 @@ constexpr int STW = 64, STH = 64;
 template <int K> struct SynthTile : TileDims<K, STW, STH> {
     static constexpr int XW = TileDims<K, STW, STH>::W, XH = TileDims<K, STW, STH>::H, XP = TileDims<K, STW, STH>::P;
 };
-
-// Four consecutive activations as floats (16-byte / 8-byte aligned vector load).
-__device__ __forceinline__ float4 load_vec4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
-__device__ __forceinline__ float4 load_vec4(const __half *p) {
-    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
-    const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&q.x));
-    const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&q.y));
-    return make_float4(a.x, a.y, b.x, b.y);
-}
-__device__ __forceinline__ float4 load_vec4(const __nv_bfloat16 *p) {
-    const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p));
-    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.x));
-    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&q.y));
-    return make_float4(a.x, a.y, b.x, b.y);
-}
 
 // Stage the STW x STH pixel tile at (y0, x0) of plane `xp` with halo R; zero outside the image.  When the
 // row length is a multiple of 4 the tile's own columns come as vector loads of 4 pixels (they are then
