@@ -276,8 +276,22 @@ __device__ __forceinline__ void stage_pixels(const T *__restrict__ xp, int H, in
 
 // Proposition 2 for the 4 x 4 pixel block with origin (Y0, X0), both multiples of 4, of plane p: level 1
 // contributes 2 x 2 coefficients per subband, level 2 one coefficient whose signs vary inside the block, every
-// deeper level one coefficient with a block-wide sign.
-__device__ __forceinline__ void block_synthesis(const LevelPtrs &lv, int L, size_t p, int Y0, int X0, float (&a)[4][4]) {
+// deeper level one coefficient with a block-wide sign.  The level-1 and level-2 coefficients are fetched first
+// (load_z12) so that their global-memory latency runs behind the block's convolution.
+struct Z12 {
+    float z1[2][2][4];  // [ci][cj][subband]
+    float z2[4];
+};
+__device__ __forceinline__ Z12 load_z12(const LevelPtrs &lv, int L, size_t p, int Y0, int X0) {
+    Z12 z;
+#pragma unroll
+    for (int ci = 0; ci < 2; ++ci)
+#pragma unroll
+        for (int cj = 0; cj < 2; ++cj)
+#pragma unroll
+            for (int sb = 0; sb < 4; ++sb) z.z1[ci][cj][sb] = 0.f;
+#pragma unroll
+    for (int sb = 0; sb < 4; ++sb) z.z2[sb] = 0.f;
     if (L >= 1) {
         const int Hl = lv.Hl[0], Wl = lv.Wl[0];
         const size_t S = (size_t)Hl * Wl;
@@ -287,15 +301,35 @@ __device__ __forceinline__ void block_synthesis(const LevelPtrs &lv, int L, size
 #pragma unroll
             for (int cj = 0; cj < 2; ++cj) {
                 const int i = (Y0 >> 1) + ci, j = (X0 >> 1) + cj;
-                if (i < Hl && j < Wl) {
+                if (i < Hl && j < Wl) {  // coefficients beyond the grid only feed pixels beyond the image
                     const float *q = zp + (size_t)i * Wl + j;
-                    const float ll = __ldg(q), lh = __ldg(q + S), hl = __ldg(q + 2 * S), hh = __ldg(q + 3 * S);
-                    const float pp = ll + lh, pm = ll - lh, qp = hl + hh, qm = hl - hh;
-                    a[2 * ci][2 * cj] = fmaf(0.5f, pp + qp, a[2 * ci][2 * cj]);
-                    a[2 * ci][2 * cj + 1] = fmaf(0.5f, pp - qp, a[2 * ci][2 * cj + 1]);
-                    a[2 * ci + 1][2 * cj] = fmaf(0.5f, pm + qm, a[2 * ci + 1][2 * cj]);
-                    a[2 * ci + 1][2 * cj + 1] = fmaf(0.5f, pm - qm, a[2 * ci + 1][2 * cj + 1]);
+#pragma unroll
+                    for (int sb = 0; sb < 4; ++sb) z.z1[ci][cj][sb] = __ldg(q + sb * S);
                 }
+            }
+    }
+    if (L >= 2) {
+        const int Wl = lv.Wl[1];
+        const size_t S = (size_t)lv.Hl[1] * Wl;
+        const float *q = lv.z[1] + p * 4 * S + (size_t)(Y0 >> 2) * Wl + (X0 >> 2);
+#pragma unroll
+        for (int sb = 0; sb < 4; ++sb) z.z2[sb] = __ldg(q + sb * S);
+    }
+    return z;
+}
+__device__ __forceinline__ void block_synthesis(const LevelPtrs &lv, int L, size_t p, int Y0, int X0, const Z12 &z,
+                                                float (&a)[4][4]) {
+    if (L >= 1) {
+#pragma unroll
+        for (int ci = 0; ci < 2; ++ci)
+#pragma unroll
+            for (int cj = 0; cj < 2; ++cj) {
+                const float ll = z.z1[ci][cj][0], lh = z.z1[ci][cj][1], hl = z.z1[ci][cj][2], hh = z.z1[ci][cj][3];
+                const float pp = ll + lh, pm = ll - lh, qp = hl + hh, qm = hl - hh;
+                a[2 * ci][2 * cj] = fmaf(0.5f, pp + qp, a[2 * ci][2 * cj]);
+                a[2 * ci][2 * cj + 1] = fmaf(0.5f, pp - qp, a[2 * ci][2 * cj + 1]);
+                a[2 * ci + 1][2 * cj] = fmaf(0.5f, pm + qm, a[2 * ci + 1][2 * cj]);
+                a[2 * ci + 1][2 * cj + 1] = fmaf(0.5f, pm - qm, a[2 * ci + 1][2 * cj + 1]);
             }
     }
     if (L >= 2) {
@@ -308,10 +342,7 @@ __device__ __forceinline__ void block_synthesis(const LevelPtrs &lv, int L, size
             deep += synth_term(__ldg(q), __ldg(q + S), __ldg(q + 2 * S), __ldg(q + 3 * S), (Y0 >> (l - 1)) & 1,
                                (X0 >> (l - 1)) & 1, scale);
         }
-        const int Wl = lv.Wl[1];
-        const size_t S = (size_t)lv.Hl[1] * Wl;
-        const float *q = lv.z[1] + p * 4 * S + (size_t)(Y0 >> 2) * Wl + (X0 >> 2);
-        const float ll = __ldg(q), lh = __ldg(q + S), hl = __ldg(q + 2 * S), hh = __ldg(q + 3 * S);
+        const float ll = z.z2[0], lh = z.z2[1], hl = z.z2[2], hh = z.z2[3];
         const float pp = ll + lh, pm = ll - lh, qp = hl + hh, qm = hl - hh;
         float t2[2][2];
         t2[0][0] = fmaf(0.25f, pp + qp, deep);
@@ -385,8 +416,9 @@ synth_fwd_kernel(const T *__restrict__ x, int H, int W, int C, int L, const floa
     for (int r = 0; r < 4; ++r)
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) acc[r][cc] = bias;
+    const Z12 z = load_z12(lv, L, (size_t)p, Y0, X0);
     block_conv<K, S::XP>(Xs, 4 * ty, 4 * tx, wr, acc);
-    block_synthesis(lv, L, (size_t)p, Y0, X0, acc);
+    block_synthesis(lv, L, (size_t)p, Y0, X0, z, acc);
     store_block<T>(out + (size_t)p * H * W, H, W, Y0, X0, acc);
 }
 
@@ -539,7 +571,8 @@ synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W,
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) acc[r][cc] = 0.f;
         block_conv<K, S::XP>(Gs, 4 * ty, 4 * tx, wf, acc);
-        block_synthesis(lv, L, p, Y0, X0, acc);
+        const Z12 z = load_z12(lv, L, p, Y0, X0);  // (fetching these ahead of the conv costs spills at 80 registers)
+        block_synthesis(lv, L, p, Y0, X0, z, acc);
         store_block<T>(dx + p * H * W, H, W, Y0, X0, acc);
     }
 #pragma unroll
