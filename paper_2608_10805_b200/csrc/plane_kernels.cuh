@@ -264,17 +264,11 @@ __device__ __forceinline__ PatchD decode_patch(const Geom &g, const int *off, in
     }
     return p;
 }
+// The 4 x 4 pixels of a patch (zero where the patch leaves the image or the plane slot is not in use).
 template <typename T, bool RAW>
-__device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD &p0_, const T *__restrict__ gsrc,
-                                          int nvalid, int d0 = 0, int d1 = 0, int d2 = 0) {
-    if (p0_.meta >= 0) return;
-    PatchD p = p0_;  // d0/d1/d2 shift the x / level-1 / level-2 targets to another set of arrays (grad_out side)
-    p.xi += d0;
-    p.yi += d1;
-    p.y2 += d2;
+__device__ __forceinline__ void load_patch(const Geom &g, const PatchD &p, const T *__restrict__ gsrc, int nvalid,
+                                           float (&a)[4][4]) {
     const int slot = p.meta & 0xff, nrows = (p.meta >> 8) & 7;
-    const int p0 = g.pitch[0], p1 = g.pitch[1], sub1 = g.rows[1] * p1, sub2 = g.rows[2] * g.pitch[2], W = g.W;
-    float a[4][4];
 #pragma unroll
     for (int rr = 0; rr < 4; ++rr)
 #pragma unroll
@@ -283,8 +277,19 @@ __device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD
         const T *pa = gsrc + slot * (g.H * g.W) + p.so;  // the unit's planes are contiguous
 #pragma unroll
         for (int rr = 0; rr < 4; ++rr)
-            if (rr < nrows) ld4<T, RAW>(pa + rr * W, a[rr]);
+            if (rr < nrows) ld4<T, RAW>(pa + rr * g.W, a[rr]);
     }
+}
+// x, level 1 and level 2 of one patch into the haloed arrays; d0/d1/d2 shift the targets to another set of
+// arrays (grad_out side).
+__device__ __forceinline__ void store_patch(float *sm, const Geom &g, const PatchD &p0_, const float (&a)[4][4], int d0,
+                                            int d1, int d2) {
+    PatchD p = p0_;
+    p.xi += d0;
+    p.yi += d1;
+    p.y2 += d2;
+    const int nrows = (p.meta >> 8) & 7;
+    const int p0 = g.pitch[0], p1 = g.pitch[1], sub1 = g.rows[1] * p1, sub2 = g.rows[2] * g.pitch[2];
 #pragma unroll
     for (int rr = 0; rr < 4; ++rr) {
         if (rr < nrows) {
@@ -310,6 +315,26 @@ __device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD
     sm[p.y2 + sub2] = h2.lh;
     sm[p.y2 + 2 * sub2] = h2.hl;
     sm[p.y2 + 3 * sub2] = h2.hh;
+}
+template <typename T, bool RAW>
+__device__ __forceinline__ void run_patch(float *sm, const Geom &g, const PatchD &p, const T *__restrict__ gsrc,
+                                          int nvalid, int d0 = 0, int d1 = 0, int d2 = 0) {
+    if (p.meta >= 0) return;
+    float a[4][4];
+    load_patch<T, RAW>(g, p, gsrc, nvalid, a);
+    store_patch(sm, g, p, a, d0, d1, d2);
+}
+// The same patch of two tensors (x and grad_out): both sets of loads are issued before either is used, so
+// their global-memory latencies overlap.
+template <typename T, bool RAW>
+__device__ __forceinline__ void run_patch_pair(float *sm, const Geom &g, const PatchD &p, const T *__restrict__ xsrc,
+                                               const T *__restrict__ gsrc, int nvalid, int d0, int d1, int d2) {
+    if (p.meta >= 0) return;
+    float a[4][4], b[4][4];
+    load_patch<T, RAW>(g, p, xsrc, nvalid, a);
+    load_patch<T, RAW>(g, p, gsrc, nvalid, b);
+    store_patch(sm, g, p, a, 0, 0, 0);
+    store_patch(sm, g, p, b, d0, d1, d2);
 }
 
 struct ItemD {    // one 4 x TH conv tile
@@ -1106,10 +1131,8 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             }
         } else if (hoist_patch) {
             const size_t po = ((size_t)b * g.C + c) * HW;
-            run_patch<T, false>(sm, g, patch0, x + po, nvalid);
-            run_patch<T, false>(sm, g, patch0, go + po, nvalid, dA0, dA1, dA2);
-            run_patch<T, false>(sm, g, patch1, x + po, nvalid);
-            run_patch<T, false>(sm, g, patch1, go + po, nvalid, dA0, dA1, dA2);
+            run_patch_pair<T, false>(sm, g, patch0, x + po, go + po, nvalid, dA0, dA1, dA2);
+            run_patch_pair<T, false>(sm, g, patch1, x + po, go + po, nvalid, dA0, dA1, dA2);
             lnext = 3;
         } else {
             lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, tid, nthr);
