@@ -243,13 +243,18 @@ template <int K> struct SynthTile : TileDims<K, STW, STH> {
     static constexpr int XW = TileDims<K, STW, STH>::W, XH = TileDims<K, STW, STH>::H, XP = TileDims<K, STW, STH>::P;
 };
 
-// Stage the STW x STH pixel tile at (y0, x0) of plane `xp` with halo R; zero outside the image.  When the
-// row length is a multiple of 4 the tile's own columns come as vector loads of 4 pixels (they are then
-// either all inside the image or all outside) and only the 2R halo columns go element by element.
+// Stage the STW x STH pixel tile at (y0, x0) of plane p of tensor `base` ([P][H][W], 16-byte aligned) with halo
+// R; zero outside the image.  When the row length is a multiple of 4 the tile's own columns come as vector loads
+// of 4 pixels (they are then either all inside the image or all outside) and only the 2R halo columns go element
+// by element.  Otherwise rows start at arbitrary element offsets: the tile is zeroed and then filled from the
+// aligned 4-element chunks of the whole tensor that overlap each tile row, every element placed on its own
+// (chunks may begin in the previous row or end in the next one; `total` = elements in the tensor bounds them).
 template <typename T, int K>
-__device__ __forceinline__ void stage_pixels(const T *__restrict__ xp, int H, int W, int y0, int x0,
-                                             float (*Xs)[SynthTile<K>::XP]) {
+__device__ __forceinline__ void stage_pixels(const T *__restrict__ base, size_t p, size_t total, int H, int W, int y0,
+                                             int x0, float (*Xs)[SynthTile<K>::XP]) {
     using S = SynthTile<K>;
+    const size_t plane0 = p * (size_t)H * W;
+    const T *xp = base + plane0;
     if ((W & 3) == 0) {
         for (int e = threadIdx.x; e < S::XH * (STW / 4); e += NTHREADS) {
             const int ly = e / (STW / 4), j = e - ly * (STW / 4);
@@ -267,10 +272,32 @@ __device__ __forceinline__ void stage_pixels(const T *__restrict__ xp, int H, in
         }
         return;
     }
-    for (int e = threadIdx.x; e < S::XH * S::XP; e += NTHREADS) {
-        const int ly = e / S::XP, lx = e - ly * S::XP;
-        const int yy = y0 + ly - S::R, xx = x0 + lx - S::R;
-        Xs[ly][lx] = (yy >= 0 && yy < H && xx >= 0 && xx < W) ? ldf(xp + (size_t)yy * W + xx) : 0.f;
+    float4 *z = reinterpret_cast<float4 *>(&Xs[0][0]);
+    for (int e = threadIdx.x; e < S::XH * S::XP / 4; e += NTHREADS) z[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+    constexpr int CH = (S::XW + 3) / 4 + 1;  // aligned chunks that can overlap one tile row
+    const int xa = x0 - S::R < 0 ? 0 : x0 - S::R;                    // first image column the tile needs
+    const int xb = x0 + STW + S::R > W ? W : x0 + STW + S::R;        // one past the last
+    for (int e = threadIdx.x; e < S::XH * CH; e += NTHREADS) {
+        const int ly = e / CH, k = e - ly * CH;
+        const int yy = y0 + ly - S::R;
+        if (yy < 0 || yy >= H || xa >= xb) continue;
+        const size_t row0 = plane0 + (size_t)yy * W;               // tensor-wide index of the row's first element
+        const size_t c = ((row0 + xa) >> 2) + k;                    // aligned chunk
+        if (4 * c >= row0 + xb) continue;
+        float v[4];
+        if (4 * c + 3 < total) {
+            const float4 t = load_vec4(base + 4 * c);
+            v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = 4 * c + i < total ? ldf(base + 4 * c + i) : 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const long long col = (long long)(4 * c + i) - (long long)row0;  // image column of this element
+            if (col >= xa && col < xb) Xs[ly][(int)col - x0 + S::R] = v[i];
+        }
     }
 }
 
@@ -397,7 +424,7 @@ synth_fwd_kernel(const T *__restrict__ x, int H, int W, int C, int L, const floa
     __shared__ __align__(16) float Xs[S::XH][S::XP];
     const int p = blockIdx.x, c = p % C;
     const int x0 = blockIdx.y * STW, y0 = blockIdx.z * STH;
-    stage_pixels<T, K>(x + (size_t)p * H * W, H, W, y0, x0, Xs);
+    stage_pixels<T, K>(x, (size_t)p, (size_t)gridDim.x * H * W, H, W, y0, x0, Xs);
     // folded weights (Eq. 8) go through shared memory once, then live in registers
     __shared__ float Ws[K * K + 1];
     const float sc = __ldg(s0 + c);
@@ -550,8 +577,8 @@ synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W,
     for (int b = part; b < B; b += bsplit) {
         const size_t p = (size_t)b * C + c;
         __syncthreads();
-        stage_pixels<T, K>(x + p * H * W, H, W, y0, x0, Xs);
-        stage_pixels<T, K>(g + p * H * W, H, W, y0, x0, Gs);
+        stage_pixels<T, K>(x, p, (size_t)B * C * H * W, H, W, y0, x0, Xs);
+        stage_pixels<T, K>(g, p, (size_t)B * C * H * W, H, W, y0, x0, Gs);
         __syncthreads();
         if (!live) continue;
         // weight gradient: the block's 16 upstream values (zero outside the image) against the shifted x window
