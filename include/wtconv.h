@@ -176,9 +176,12 @@ wtconv_status wtconv_backward_static(const wtconv_desc *desc, const void *x, con
  * copies to overlap; they must stay valid until the stream reaches this point).
  * Every h_* pointer is a HOST pointer with the layouts above; `workspace` is DEVICE scratch of
  * at least wtconv_step_host_workspace_bytes.  h_b0 / h_grad_b0 may both be NULL.
- * The forward result is copied back on a library-internal stream (one per device, created on the first
- * call) while grad_out is still being uploaded; `stream` waits for that copy, so everything is complete
- * when `stream` reaches this point.  The first call on a device must not happen inside a stream capture. */
+ * Copies overlap the kernels: large batches are processed in up to eight chunks whose uploads, kernels and
+ * downloads run on `stream` and two library-internal streams (per device, created on the first call), and the
+ * chunks' parameter gradients are added in chunk order; small ones send the forward result back while grad_out
+ * is still being uploaded.  `stream` waits for the internal streams, so everything is complete when `stream`
+ * reaches this point.  The first call on a device must not happen inside a stream capture, and two calls
+ * on one device must not overlap in time (they would share the internal streams' ordering, not their data). */
 wtconv_status wtconv_step_host_workspace_bytes(const wtconv_desc *desc, size_t *bytes);
 wtconv_status wtconv_step_host(const wtconv_desc *desc, const void *h_x, const void *h_grad_out,
                                const float *h_w0, const float *h_s0, const float *h_b0,

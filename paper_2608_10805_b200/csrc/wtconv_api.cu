@@ -296,16 +296,36 @@ wtconv_status static_scratch_for_current_device(void **out) {
     return WTCONV_OK;
 }
 
+// wtconv_step_host splits the batch into chunks so that uploads, kernels and downloads of different chunks overlap.
+constexpr int STEP_MAX_CHUNKS = 8;
+int pick_step_chunks(const wtconv_desc *d) {
+    const size_t per_image = (size_t)d->C * d->H * d->W * elem_bytes(d->dtype);
+    for (int n = STEP_MAX_CHUNKS; n >= 2; n /= 2)
+        if (d->B % n == 0 && d->B / n >= 4 && ((size_t)(d->B / n) * per_image) % 16 == 0 &&
+            (size_t)(d->B / n) * per_image >= ((size_t)4 << 20))
+            return n;
+    return 1;
+}
+// dst[i] = sum over chunks of src[c * stride + i], in chunk order (deterministic).
+__global__ void sum_chunks_kernel(float *__restrict__ dst, const float *__restrict__ src, size_t n, int nch, size_t stride) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float a = src[i];
+    for (int c = 1; c < nch; ++c) a += src[(size_t)c * stride + i];
+    dst[i] = a;
+}
+
 // Internal copy stream of wtconv_step_host, one per device, created on first use and kept for the process.
 std::mutex g_side_mutex;
-cudaStream_t g_side_stream[MAX_DEVICES] = {};
-wtconv_status side_stream_for_current_device(cudaStream_t *out) {
+cudaStream_t g_side_stream[MAX_DEVICES][2] = {};  // [0] downloads, [1] uploads
+wtconv_status side_stream_for_current_device(cudaStream_t *out, int which = 0) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return WTCONV_ERR_CUDA;
     std::lock_guard<std::mutex> lock(g_side_mutex);
-    if (!g_side_stream[dev] && cudaStreamCreateWithFlags(&g_side_stream[dev], cudaStreamNonBlocking) != cudaSuccess)
+    if (!g_side_stream[dev][which] &&
+        cudaStreamCreateWithFlags(&g_side_stream[dev][which], cudaStreamNonBlocking) != cudaSuccess)
         return WTCONV_ERR_CUDA;
-    *out = g_side_stream[dev];
+    *out = g_side_stream[dev][which];
     return WTCONV_OK;
 }
 
@@ -421,7 +441,8 @@ wtconv_status wtconv_step_host_workspace_bytes(const wtconv_desc *d, size_t *byt
     ParamSizes ps = param_sizes(d);
     const size_t par = align_up(ps.w0) + 2 * align_up(ps.s0) + align_up(ps.wl) + align_up(ps.sl);
     size_t f = fwd_ws_bytes(d), b = bwd_ws_bytes(d);
-    *bytes = 4 * act + 2 * par + (f > b ? f : b);
+    // parameters, their gradients, and one more gradient set per batch chunk of the pipelined step
+    *bytes = 4 * act + (2 + STEP_MAX_CHUNKS) * par + (f > b ? f : b);
     return WTCONV_OK;
 }
 
@@ -472,6 +493,83 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
         cudaEvent_t a, b;
         ~EventGuard() { cudaEventDestroy(a); cudaEventDestroy(b); }
     } guard = {fwd_done, out_home};
+    const float *b0p = h_b0 ? b0 : nullptr;
+    const int nch = pick_step_chunks(d);
+    if (nch > 1) {
+        // Pipelined step: chunk c's upload and kernels run on `stream`, its results travel back on the internal
+        // stream while chunk c+1 is uploaded.  Every chunk leaves its own parameter gradients; they are added
+        // in chunk order at the end.
+        const size_t par_bytes = (size_t)((char *)gsl + align_up(ps.sl) - (char *)gw0);  // one gradient set
+        char *chunk_grads = p;
+        p += (size_t)STEP_MAX_CHUNKS * par_bytes;
+        const size_t rest_c = workspace_bytes - (size_t)(p - (char *)workspace);
+        wtconv_desc dc = *d;
+        dc.B = d->B / nch;
+        const size_t cb = act_raw / nch;
+        h2d(w0, h_w0, ps.w0);
+        h2d(s0, h_s0, ps.s0);
+        if (h_b0) h2d(b0, h_b0, ps.s0);
+        h2d(wl, h_wl, ps.wl);
+        h2d(sl, h_sl, ps.sl);
+        // events: [0..nch) chunk computed, [nch] downloads done, [nch+1] stream position at entry,
+        // [nch+2 .. 2 nch+2) chunk uploaded
+        constexpr int NEV = 2 * STEP_MAX_CHUNKS + 2;
+        cudaEvent_t ev[NEV] = {};
+        struct EventsGuard {
+            cudaEvent_t *e;
+            ~EventsGuard() { for (int i = 0; i < NEV; ++i) if (e[i]) cudaEventDestroy(e[i]); }
+        } eguard = {ev};
+        for (int c = 0; c < 2 * nch + 2 && ok; ++c) ok = cudaEventCreateWithFlags(&ev[c], cudaEventDisableTiming) == cudaSuccess;
+        cudaStream_t up = nullptr;
+        if (ok && side_stream_for_current_device(&up, 1) != WTCONV_OK) ok = false;
+        if (!ok) return WTCONV_ERR_CUDA;
+        // uploads run on their own stream (behind whatever `stream` holds at entry), so that chunk c+1 arrives
+        // while chunk c is being computed
+        ok = ok && cudaEventRecord(ev[nch + 1], cs) == cudaSuccess && cudaStreamWaitEvent(up, ev[nch + 1], 0) == cudaSuccess;
+        for (int c = 0; c < nch && ok; ++c) {
+            const size_t o = (size_t)c * cb;
+            ok = ok && cudaMemcpyAsync(dx_ + o, (const char *)h_x + o, cb, cudaMemcpyHostToDevice, up) == cudaSuccess;
+            ok = ok && cudaMemcpyAsync(dg + o, (const char *)h_g + o, cb, cudaMemcpyHostToDevice, up) == cudaSuccess;
+            ok = ok && cudaEventRecord(ev[nch + 2 + c], up) == cudaSuccess;
+        }
+        if (!ok) {  // nothing of this step may outlive the caller's stream position
+            if (cudaEventRecord(ev[nch], up) == cudaSuccess) cudaStreamWaitEvent(cs, ev[nch], 0);
+            return WTCONV_ERR_CUDA;
+        }
+        for (int c = 0; c < nch; ++c) {
+            const size_t o = (size_t)c * cb;
+            ok = ok && cudaStreamWaitEvent(cs, ev[nch + 2 + c], 0) == cudaSuccess;
+            if (!ok) break;
+            char *gq = chunk_grads + (size_t)c * par_bytes;  // same layout as the final gradient set
+            float *cgw0 = (float *)gq, *cgs0 = (float *)(gq + ((char *)gs0 - (char *)gw0)),
+                  *cgb0 = (float *)(gq + ((char *)gb0 - (char *)gw0)), *cgwl = (float *)(gq + ((char *)gwl - (char *)gw0)),
+                  *cgsl = (float *)(gq + ((char *)gsl - (char *)gw0));
+            st = wtconv_forward(&dc, dx_ + o, w0, s0, b0p, wl, sl, dout + o, p, rest_c, stream);
+            if (st == WTCONV_OK)
+                st = wtconv_backward(&dc, dx_ + o, dg + o, w0, s0, b0p, wl, sl, dgx + o, cgw0, cgs0, h_b0 ? cgb0 : nullptr,
+                                     cgwl, cgsl, p, rest_c, stream);
+            if (st != WTCONV_OK) break;
+            ok = ok && cudaEventRecord(ev[c], cs) == cudaSuccess;
+            ok = ok && cudaStreamWaitEvent(side, ev[c], 0) == cudaSuccess;
+            if (ok) ok = cudaMemcpyAsync((char *)h_out + o, dout + o, cb, cudaMemcpyDeviceToHost, side) == cudaSuccess;
+            if (ok) ok = cudaMemcpyAsync((char *)h_gx + o, dgx + o, cb, cudaMemcpyDeviceToHost, side) == cudaSuccess;
+        }
+        // join first, so that `stream` ends after both internal streams whatever happened above (every upload
+        // event has either been waited for by `stream` or precedes the last one, which is waited for here)
+        bool joined = cudaStreamWaitEvent(cs, ev[nch + 2 + nch - 1], 0) == cudaSuccess &&
+                      cudaEventRecord(ev[nch], side) == cudaSuccess && cudaStreamWaitEvent(cs, ev[nch], 0) == cudaSuccess;
+        if (st != WTCONV_OK) return st;
+        if (!ok || !joined) return WTCONV_ERR_CUDA;
+        const size_t nfl = par_bytes / sizeof(float);
+        sum_chunks_kernel<<<(unsigned)((nfl + 255) / 256), 256, 0, cs>>>(gw0, (const float *)chunk_grads, nfl, nch, nfl);
+        if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
+        d2h(h_gw0, gw0, ps.w0);
+        d2h(h_gs0, gs0, ps.s0);
+        if (h_b0) d2h(h_gb0, gb0, ps.s0);
+        d2h(h_gwl, gwl, ps.wl);
+        d2h(h_gsl, gsl, ps.sl);
+        return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
+    }
     h2d(dx_, h_x, act_raw);
     h2d(w0, h_w0, ps.w0);
     h2d(s0, h_s0, ps.s0);
@@ -479,7 +577,6 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     h2d(wl, h_wl, ps.wl);
     h2d(sl, h_sl, ps.sl);
     if (!ok) return WTCONV_ERR_CUDA;
-    const float *b0p = h_b0 ? b0 : nullptr;
     st = wtconv_forward(d, dx_, w0, s0, b0p, wl, sl, dout, p, rest, stream);
     if (st != WTCONV_OK) return st;
     ok = ok && cudaEventRecord(fwd_done, cs) == cudaSuccess;

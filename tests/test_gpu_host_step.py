@@ -16,6 +16,7 @@ pytestmark = pytest.mark.gpu
     (Workload("host_plane", 3, 4, 28, 28, 5, 2, "f32", 51), True),
     (Workload("host_bf16", 4, 6, 14, 14, 5, 1, "bf16", 52), False),
     (Workload("host_tiled", 1, 2, 90, 75, 3, 2, "f32", 53), False),
+    (Workload("host_chunked", 64, 16, 56, 56, 5, 3, "f32", 54), True),   # large enough for the chunked pipeline
 ], ids=lambda v: v.name if isinstance(v, Workload) else str(v))
 def test_host_step_matches_oracle(wl, bias):
     tdt = wt.DTYPE_NAMES[wl.dtype]
