@@ -20,6 +20,10 @@ constexpr int TW = 32;       // level kernels: tile width in coefficients
 constexpr int TH = 32;       // level kernels: tile height in coefficients
 constexpr int NTHREADS = 256;
 
+// Grids are one-dimensional and plane-major: the tiles of one plane (or of one channel's batch slice) are
+// neighbours in launch order, so the halo a tile shares with the next one is still in L2 when that one runs.
+__host__ __device__ inline int tiles_of(int n, int t) { return (n + t - 1) / t; }
+
 // Shared-memory tile of TWc x THc outputs with halo R = K/2.  Every thread computes a 4 x 4 output block; its
 // window starts at a multiple of four floats, so window rows are read as NQ aligned float4 loads, and the pitch
 // P leaves room for the last thread's last load.
@@ -197,8 +201,9 @@ level_fwd_kernel(const Tin *__restrict__ Xprev, int Hp, int Wp, int Hl, int Wl, 
     constexpr int KK = K * K;
     __shared__ __align__(16) float Ys[4][D::H][D::P];
     __shared__ float Ws[4][KK];
-    const int p = blockIdx.x, c = p % C;
-    const int j0 = blockIdx.y * TW, i0 = blockIdx.z * TH;
+    const int ntx = tiles_of(Wl, TW), ntile = ntx * tiles_of(Hl, TH);
+    const int p = blockIdx.x / ntile, tile = blockIdx.x - p * ntile, c = p % C;
+    const int j0 = (tile % ntx) * TW, i0 = (tile / ntx) * TH;
     stage_subbands<Tin, K>(Xprev + (size_t)p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
     if (threadIdx.x < 4 * KK)  // Eq. 8
         Ws[threadIdx.x / KK][threadIdx.x % KK] = __ldg(s + c * 4 + threadIdx.x / KK) * __ldg(w + (size_t)c * 4 * KK + threadIdx.x);
@@ -422,9 +427,10 @@ synth_fwd_kernel(const T *__restrict__ x, int H, int W, int C, int L, const floa
                  const float *__restrict__ s0, const float *__restrict__ b0, LevelPtrs lv, T *__restrict__ out) {
     using S = SynthTile<K>;
     __shared__ __align__(16) float Xs[S::XH][S::XP];
-    const int p = blockIdx.x, c = p % C;
-    const int x0 = blockIdx.y * STW, y0 = blockIdx.z * STH;
-    stage_pixels<T, K>(x, (size_t)p, (size_t)gridDim.x * H * W, H, W, y0, x0, Xs);
+    const int ntx = tiles_of(W, STW), ntile = ntx * tiles_of(H, STH);
+    const int p = blockIdx.x / ntile, tile = blockIdx.x - p * ntile, c = p % C;
+    const int x0 = (tile % ntx) * STW, y0 = (tile / ntx) * STH;
+    stage_pixels<T, K>(x, (size_t)p, (size_t)(gridDim.x / ntile) * H * W, H, W, y0, x0, Xs);
     // folded weights (Eq. 8) go through shared memory once, then live in registers
     __shared__ float Ws[K * K + 1];
     const float sc = __ldg(s0 + c);
@@ -482,8 +488,10 @@ level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, i
     float (*Ds)[D::H][D::P] = reinterpret_cast<float (*)[D::H][D::P]>(lsm + 4 * D::H * D::P);
     float (*red)[KK] = reinterpret_cast<float (*)[KK]>(lsm + 8 * D::H * D::P);
     float (*Ws)[KK] = reinterpret_cast<float (*)[KK]>(lsm + 8 * D::H * D::P + 8 * KK);
-    const int c = blockIdx.x / bsplit, part = blockIdx.x - c * bsplit;
-    const int j0 = blockIdx.y * TW, i0 = blockIdx.z * TH;
+    const int ntx = tiles_of(Wl, TW), ntile = ntx * tiles_of(Hl, TH);
+    const int cp = blockIdx.x / ntile, tile = blockIdx.x - cp * ntile;
+    const int c = cp / bsplit, part = cp - c * bsplit;
+    const int j0 = (tile % ntx) * TW, i0 = (tile / ntx) * TH;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = threadIdx.x >> 6, tx = threadIdx.x & 7, ty = (threadIdx.x >> 3) & 7;
     const int I0 = i0 + 4 * ty, J0 = j0 + 4 * tx;
@@ -537,8 +545,8 @@ level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, i
         if (lane == 0) red[warp][t] = v;
     }
     __syncthreads();
-    const int nparts = gridDim.y * gridDim.z * bsplit;
-    const int pidx = (blockIdx.z * gridDim.y + blockIdx.y) * bsplit + part;
+    const int nparts = ntile * bsplit;
+    const int pidx = tile * bsplit + part;
     for (int e = threadIdx.x; e < 4 * KK; e += NTHREADS) {
         int sb = e / KK, t = e - sb * KK;
         partials[(((size_t)c * nparts + pidx) * 4 + sb) * KK + t] = red[2 * sb][t] + red[2 * sb + 1][t];
@@ -561,8 +569,10 @@ synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W,
     __shared__ __align__(16) float Xs[S::XH][S::XP];
     __shared__ __align__(16) float Gs[S::XH][S::XP];
     __shared__ float red[8][KK + 1];
-    const int c = blockIdx.x / bsplit, part = blockIdx.x - c * bsplit;
-    const int x0 = blockIdx.y * STW, y0 = blockIdx.z * STH;
+    const int ntx = tiles_of(W, STW), ntile = ntx * tiles_of(H, STH);
+    const int cp = blockIdx.x / ntile, tile = blockIdx.x - cp * ntile;
+    const int c = cp / bsplit, part = cp - c * bsplit;
+    const int x0 = (tile % ntx) * STW, y0 = (tile / ntx) * STH;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int X0 = x0 + 4 * tx, Y0 = y0 + 4 * ty;
@@ -612,13 +622,13 @@ synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W,
         if (lane == 0) red[warp][KK] = v;
     }
     __syncthreads();
-    const int nparts = gridDim.y * gridDim.z * bsplit;
-    const int pidx = (blockIdx.z * gridDim.y + blockIdx.y) * bsplit + part;
-    for (int t = threadIdx.x; t < KK + 1; t += NTHREADS) {
+    const int nparts = ntile * bsplit;
+    const int pidx = tile * bsplit + part;
+    for (int e = threadIdx.x; e < KK + 1; e += NTHREADS) {
         float v = 0.f;
 #pragma unroll
-        for (int wi = 0; wi < 8; ++wi) v += red[wi][t];
-        partials[((size_t)c * nparts + pidx) * (KK + 1) + t] = v;
+        for (int wi = 0; wi < 8; ++wi) v += red[wi][e];
+        partials[((size_t)c * nparts + pidx) * (KK + 1) + e] = v;
     }
 }
 

@@ -130,7 +130,7 @@ wtconv_status tiled_forward(const wtconv_desc *d, const T *x, const float *w0, c
         const int Hp = pl.sh.Hs[l - 1], Wp = pl.sh.Ws[l - 1], Hl = pl.sh.Hs[l], Wl = pl.sh.Ws[l];
         float *Z = (float *)(ws + pl.z_off[l - 1]);
         float *Xl = (l < d->L) ? (float *)(ws + pl.xc_off[l - 1]) : nullptr;
-        dim3 grid(pl.P, cdiv(Wl, TW), cdiv(Hl, TH));
+        dim3 grid((unsigned)((size_t)pl.P * cdiv(Wl, TW) * cdiv(Hl, TH)));  // plane-major
         const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
         if (l == 1)
             level_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, Hp, Wp, Hl, Wl, C, wq, sq, Z, Xl);
@@ -141,7 +141,7 @@ wtconv_status tiled_forward(const wtconv_desc *d, const T *x, const float *w0, c
         lv.Hl[l - 1] = Hl;
         lv.Wl[l - 1] = Wl;
     }
-    dim3 grid(pl.P, cdiv(d->W, STW), cdiv(d->H, STH));
+    dim3 grid((unsigned)((size_t)pl.P * cdiv(d->W, STW) * cdiv(d->H, STH)));  // plane-major
     synth_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, d->H, d->W, C, d->L, w0, s0, b0, lv, out);
     return launch_status();
 }
@@ -171,7 +171,7 @@ wtconv_status tiled_backward(const wtconv_desc *d, const T *x, const T *g, const
         float *Xl = (l < d->L) ? (float *)(ws + pl.xc_off[l - 1]) : nullptr;
         float *Gl = (l < d->L) ? (float *)(ws + pl.gc_off[l - 1]) : nullptr;
         float *part = (float *)(ws + pl.partl_off[l - 1]);
-        dim3 grid(C * pl.bsplitl[l - 1], pl.txl[l - 1], pl.tyl[l - 1]);
+        dim3 grid((unsigned)((size_t)C * pl.bsplitl[l - 1] * pl.txl[l - 1] * pl.tyl[l - 1]));  // (channel, part)-major
         const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
         constexpr size_t lsmem = level_bwd_smem_bytes<K>();  // above 48 KB for k = 7: opt in
         if (l == 1) {
@@ -193,7 +193,7 @@ wtconv_status tiled_backward(const wtconv_desc *d, const T *x, const T *g, const
         ep.npl[l - 1] = pl.npl[l - 1];
     }
     float *part0 = (float *)(ws + pl.part0_off);
-    dim3 grid(C * pl.bsplit0, pl.tx0, pl.ty0);
+    dim3 grid((unsigned)((size_t)C * pl.bsplit0 * pl.tx0 * pl.ty0));  // (channel, part)-major
     synth_bwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, g, d->H, d->W, d->B, C, d->L, pl.bsplit0, w0, s0, lv, gx,
                                                       part0);
     ep.part0 = part0;
