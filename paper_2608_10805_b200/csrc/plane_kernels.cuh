@@ -162,21 +162,38 @@ __device__ __forceinline__ void build_weight_table(float *wtab, const Geom &g, i
                                                    const float *__restrict__ b0, const float *__restrict__ wl,
                                                    const float *__restrict__ sl) {
     // one table per plane slot (channel c0 + slot): [slot][class][WT_STRIDE], folded bias at [slot][0][25]
-    const int ncls = 1 + 4 * g.L;
-    for (int e = threadIdx.x; e < g.NPL * ncls * KK; e += blockDim.x) {
-        const int sc = e / KK, t = e - sc * KK, slot = sc / ncls, cls = sc - slot * ncls;
-        const int c = c0 + slot, src = flip ? (KK - 1 - t) : t;
-        float w = 0.f;
-        if (c < g.C) {
-            if (cls == 0) {
-                w = __ldg(w0 + c * KK + src) * __ldg(s0 + c);
-            } else {
-                const int l = (cls - 1) >> 2, sub = (cls - 1) & 3;
-                const size_t i = ((size_t)l * g.C + c) * 4 + sub;
-                w = __ldg(wl + i * KK + src) * __ldg(sl + i);
+    const int ncls = 1 + 4 * g.L, n = g.NPL * ncls * KK;
+    constexpr int WB = 4;
+    // four entries per step, all eight loads issued before the first product: a 16-plane unit's table has 2000
+    // entries and every block builds it, so the loads must overlap
+    for (int e0 = threadIdx.x; e0 < n; e0 += WB * blockDim.x) {
+        float wv[WB], sv[WB];
+        int dst[WB];
+#pragma unroll
+        for (int k = 0; k < WB; ++k) {
+            const int e = e0 + k * blockDim.x;
+            wv[k] = sv[k] = 0.f;
+            dst[k] = -1;
+            if (e < n) {
+                const int sc = e / KK, t = e - sc * KK, slot = sc / ncls, cls = sc - slot * ncls;
+                const int c = c0 + slot, src = flip ? (KK - 1 - t) : t;
+                dst[k] = sc * WT_STRIDE + t;
+                if (c < g.C) {
+                    if (cls == 0) {
+                        wv[k] = __ldg(w0 + c * KK + src);
+                        sv[k] = __ldg(s0 + c);
+                    } else {
+                        const int l = (cls - 1) >> 2, sub = (cls - 1) & 3;
+                        const size_t i = ((size_t)l * g.C + c) * 4 + sub;
+                        wv[k] = __ldg(wl + i * KK + src);
+                        sv[k] = __ldg(sl + i);
+                    }
+                }
             }
         }
-        wtab[sc * WT_STRIDE + t] = w;  // Eq. 8: scale folded into the weight
+#pragma unroll
+        for (int k = 0; k < WB; ++k)
+            if (dst[k] >= 0) wtab[dst[k]] = wv[k] * sv[k];  // Eq. 8: scale folded into the weight
     }
     for (int slot = threadIdx.x; slot < g.NPL; slot += blockDim.x)
         wtab[slot * ncls * WT_STRIDE + KK] = (b0 && c0 + slot < g.C) ? __ldg(s0 + c0 + slot) * __ldg(b0 + c0 + slot) : 0.f;
