@@ -72,22 +72,32 @@ __device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int H
     if ((D::R & 1) == 0 && (Wp & 3) == 0) {
         // two coefficients per step from one 4-pixel vector load per row: with an even halo and rows that are
         // multiples of four pixels a pair (j even) is aligned and lies wholly inside or wholly outside the grid
-        for (int e = threadIdx.x; e < D::H * (D::P / 2); e += NTHREADS) {
+        constexpr int NIT = (D::H * (D::P / 2) + NTHREADS - 1) / NTHREADS;
+        float4 t[NIT], u[NIT];  // all loads of a thread are issued before the first butterfly
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int e = threadIdx.x + it * NTHREADS;
             const int li = e / (D::P / 2), lj = 2 * (e - li * (D::P / 2));
             const int i = i0 + li - D::R, j = j0 + lj - D::R;
-            Haar4 h0 = {0.f, 0.f, 0.f, 0.f}, h1 = {0.f, 0.f, 0.f, 0.f};
-            if (lj < D::W && i >= 0 && i < Hl && j >= 0 && j < Wl) {
+            t[it] = u[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (e < D::H * (D::P / 2) && lj < D::W && i >= 0 && i < Hl && j >= 0 && j < Wl) {
                 const Tin *q = xp + (size_t)(2 * i) * Wp + 2 * j;
-                const float4 t = load_vec4(q);
-                float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (2 * i + 1 < Hp) u = load_vec4(q + Wp);
-                h0 = haar_butterfly(t.x, t.y, u.x, u.y);
-                h1 = haar_butterfly(t.z, t.w, u.z, u.w);
+                t[it] = load_vec4(q);
+                if (2 * i + 1 < Hp) u[it] = load_vec4(q + Wp);
             }
-            *reinterpret_cast<float2 *>(&Ys[0][li][lj]) = make_float2(h0.ll, h1.ll);
-            *reinterpret_cast<float2 *>(&Ys[1][li][lj]) = make_float2(h0.lh, h1.lh);
-            *reinterpret_cast<float2 *>(&Ys[2][li][lj]) = make_float2(h0.hl, h1.hl);
-            *reinterpret_cast<float2 *>(&Ys[3][li][lj]) = make_float2(h0.hh, h1.hh);
+        }
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int e = threadIdx.x + it * NTHREADS;
+            if (e < D::H * (D::P / 2)) {
+                const int li = e / (D::P / 2), lj = 2 * (e - li * (D::P / 2));
+                const Haar4 h0 = haar_butterfly(t[it].x, t[it].y, u[it].x, u[it].y);
+                const Haar4 h1 = haar_butterfly(t[it].z, t[it].w, u[it].z, u[it].w);
+                *reinterpret_cast<float2 *>(&Ys[0][li][lj]) = make_float2(h0.ll, h1.ll);
+                *reinterpret_cast<float2 *>(&Ys[1][li][lj]) = make_float2(h0.lh, h1.lh);
+                *reinterpret_cast<float2 *>(&Ys[2][li][lj]) = make_float2(h0.hl, h1.hl);
+                *reinterpret_cast<float2 *>(&Ys[3][li][lj]) = make_float2(h0.hh, h1.hh);
+            }
         }
         return;
     }
@@ -261,13 +271,25 @@ __device__ __forceinline__ void stage_pixels(const T *__restrict__ base, size_t 
     const size_t plane0 = p * (size_t)H * W;
     const T *xp = base + plane0;
     if ((W & 3) == 0) {
-        for (int e = threadIdx.x; e < S::XH * (STW / 4); e += NTHREADS) {
+        // all of a thread's vector loads are issued before the first one is used
+        constexpr int NIT = (S::XH * (STW / 4) + NTHREADS - 1) / NTHREADS;
+        float4 v[NIT];
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int e = threadIdx.x + it * NTHREADS;
             const int ly = e / (STW / 4), j = e - ly * (STW / 4);
             const int yy = y0 + ly - S::R, xx = x0 + 4 * j;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (yy >= 0 && yy < H && xx < W) v = load_vec4(xp + (size_t)yy * W + xx);
-            float *q = &Xs[ly][S::R + 4 * j];
-            q[0] = v.x; q[1] = v.y; q[2] = v.z; q[3] = v.w;
+            v[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (e < S::XH * (STW / 4) && yy >= 0 && yy < H && xx < W) v[it] = load_vec4(xp + (size_t)yy * W + xx);
+        }
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int e = threadIdx.x + it * NTHREADS;
+            if (e < S::XH * (STW / 4)) {
+                const int ly = e / (STW / 4), j = e - ly * (STW / 4);
+                float *q = &Xs[ly][S::R + 4 * j];
+                q[0] = v[it].x; q[1] = v[it].y; q[2] = v[it].z; q[3] = v[it].w;
+            }
         }
         for (int e = threadIdx.x; e < S::XH * (S::XP - STW); e += NTHREADS) {
             const int ly = e / (S::XP - STW), h = e - ly * (S::XP - STW);
