@@ -66,7 +66,7 @@ __device__ __forceinline__ float2 load_pair(const __nv_bfloat16 *p) {
 // from the previous carrier plane `xp` (Hp x Wp).  Positions outside the level grid are zero
 // (the depthwise conv's zero padding); pixels outside the carrier are zero (odd-size padding).
 template <typename Tin, int K>
-__device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int Hp, int Wp, int Hl, int Wl, int i0,
+__device__ __forceinline__ void stage_subbands_batched(const Tin *__restrict__ xp, int Hp, int Wp, int Hl, int Wl, int i0,
                                                int j0, float (*Ys)[LevelTile<K>::H][LevelTile<K>::P] /* [4] */) {
     using D = LevelTile<K>;
     if ((D::R & 1) == 0 && (Wp & 3) == 0) {
@@ -102,6 +102,71 @@ __device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int H
         return;
     }
     const bool even = (Wp & 1) == 0;
+    constexpr int NIT = (D::H * D::P + NTHREADS - 1) / NTHREADS;
+    float px[NIT][4];  // the 2 x 2 pixels of each of this thread's coefficients: all loads before the first butterfly
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        const int e = threadIdx.x + it * NTHREADS;
+        const int li = e / D::P, lj = e - li * D::P;
+        const int i = i0 + li - D::R, j = j0 + lj - D::R;
+        px[it][0] = px[it][1] = px[it][2] = px[it][3] = 0.f;
+        if (e < D::H * D::P && lj < D::W && i >= 0 && i < Hl && j >= 0 && j < Wl) {
+            const int y = 2 * i, x = 2 * j;
+            const bool y1 = (y + 1 < Hp);
+            const Tin *q = xp + (size_t)y * Wp + x;
+            if (even) {
+                const float2 t = load_pair(q);
+                px[it][0] = t.x; px[it][1] = t.y;
+                if (y1) { const float2 u = load_pair(q + Wp); px[it][2] = u.x; px[it][3] = u.y; }
+            } else {
+                const bool x1 = (x + 1 < Wp);
+                px[it][0] = ldf(q);
+                if (x1) px[it][1] = ldf(q + 1);
+                if (y1) { px[it][2] = ldf(q + Wp); if (x1) px[it][3] = ldf(q + Wp + 1); }
+            }
+        }
+    }
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        const int e = threadIdx.x + it * NTHREADS;
+        if (e < D::H * D::P) {
+            const int li = e / D::P, lj = e - li * D::P;
+            const Haar4 h = haar_butterfly(px[it][0], px[it][1], px[it][2], px[it][3]);
+            Ys[0][li][lj] = h.ll;
+            Ys[1][li][lj] = h.lh;
+            Ys[2][li][lj] = h.hl;
+            Ys[3][li][lj] = h.hh;
+        }
+    }
+}
+
+template <typename Tin, int K>
+__device__ __forceinline__ void stage_subbands_looped(const Tin *__restrict__ xp, int Hp, int Wp, int Hl, int Wl, int i0,
+                                               int j0, float (*Ys)[LevelTile<K>::H][LevelTile<K>::P] /* [4] */) {
+    using D = LevelTile<K>;
+    if ((D::R & 1) == 0 && (Wp & 3) == 0) {
+        // two coefficients per step from one 4-pixel vector load per row: with an even halo and rows that are
+        // multiples of four pixels a pair (j even) is aligned and lies wholly inside or wholly outside the grid
+        for (int e = threadIdx.x; e < D::H * (D::P / 2); e += NTHREADS) {
+            const int li = e / (D::P / 2), lj = 2 * (e - li * (D::P / 2));
+            const int i = i0 + li - D::R, j = j0 + lj - D::R;
+            Haar4 h0 = {0.f, 0.f, 0.f, 0.f}, h1 = {0.f, 0.f, 0.f, 0.f};
+            if (lj < D::W && i >= 0 && i < Hl && j >= 0 && j < Wl) {
+                const Tin *q = xp + (size_t)(2 * i) * Wp + 2 * j;
+                const float4 t = load_vec4(q);
+                float4 u = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (2 * i + 1 < Hp) u = load_vec4(q + Wp);
+                h0 = haar_butterfly(t.x, t.y, u.x, u.y);
+                h1 = haar_butterfly(t.z, t.w, u.z, u.w);
+            }
+            *reinterpret_cast<float2 *>(&Ys[0][li][lj]) = make_float2(h0.ll, h1.ll);
+            *reinterpret_cast<float2 *>(&Ys[1][li][lj]) = make_float2(h0.lh, h1.lh);
+            *reinterpret_cast<float2 *>(&Ys[2][li][lj]) = make_float2(h0.hl, h1.hl);
+            *reinterpret_cast<float2 *>(&Ys[3][li][lj]) = make_float2(h0.hh, h1.hh);
+        }
+        return;
+    }
+    const bool even = (Wp & 1) == 0;
     for (int e = threadIdx.x; e < D::H * D::P; e += NTHREADS) {
         const int li = e / D::P, lj = e - li * D::P;
         const int i = i0 + li - D::R, j = j0 + lj - D::R;
@@ -128,6 +193,15 @@ __device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int H
         Ys[2][li][lj] = h.hl;
         Ys[3][li][lj] = h.hh;
     }
+}
+
+// BATCH = true issues all of a thread's loads before the first use (hides the load latency, costs registers:
+// used where the kernel has them to spare); BATCH = false is the plain loop.
+template <typename Tin, int K, bool BATCH>
+__device__ __forceinline__ void stage_subbands(const Tin *__restrict__ xp, int Hp, int Wp, int Hl, int Wl, int i0,
+                                               int j0, float (*Ys)[LevelTile<K>::H][LevelTile<K>::P] /* [4] */) {
+    if (BATCH) stage_subbands_batched<Tin, K>(xp, Hp, Wp, Hl, Wl, i0, j0, Ys);
+    else stage_subbands_looped<Tin, K>(xp, Hp, Wp, Hl, Wl, i0, j0, Ys);
 }
 
 // 4 x 4 outputs of the k x k correlation with register weights; `Xs` has pitch P and the window starts at
@@ -214,7 +288,7 @@ level_fwd_kernel(const Tin *__restrict__ Xprev, int Hp, int Wp, int Hl, int Wl, 
     const int ntx = tiles_of(Wl, TW), ntile = ntx * tiles_of(Hl, TH);
     const int p = blockIdx.x / ntile, tile = blockIdx.x - p * ntile, c = p % C;
     const int j0 = (tile % ntx) * TW, i0 = (tile / ntx) * TH;
-    stage_subbands<Tin, K>(Xprev + (size_t)p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
+    stage_subbands<Tin, K, true>(Xprev + (size_t)p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
     if (threadIdx.x < 4 * KK)  // Eq. 8
         Ws[threadIdx.x / KK][threadIdx.x % KK] = __ldg(s + c * 4 + threadIdx.x / KK) * __ldg(w + (size_t)c * 4 * KK + threadIdx.x);
     __syncthreads();
@@ -265,7 +339,7 @@ template <int K> struct SynthTile : TileDims<K, STW, STH> {
 // aligned 4-element chunks of the whole tensor that overlap each tile row, every element placed on its own
 // (chunks may begin in the previous row or end in the next one; `total` = elements in the tensor bounds them).
 template <typename T, int K>
-__device__ __forceinline__ void stage_pixels(const T *__restrict__ base, size_t p, size_t total, int H, int W, int y0,
+__device__ __forceinline__ void stage_pixels_batched(const T *__restrict__ base, size_t p, size_t total, int H, int W, int y0,
                                              int x0, float (*Xs)[SynthTile<K>::XP]) {
     using S = SynthTile<K>;
     const size_t plane0 = p * (size_t)H * W;
@@ -305,6 +379,69 @@ __device__ __forceinline__ void stage_pixels(const T *__restrict__ base, size_t 
     constexpr int CH = (S::XW + 3) / 4 + 1;  // aligned chunks that can overlap one tile row
     const int xa = x0 - S::R < 0 ? 0 : x0 - S::R;                    // first image column the tile needs
     const int xb = x0 + STW + S::R > W ? W : x0 + STW + S::R;        // one past the last
+    constexpr int NIT = (S::XH * CH + NTHREADS - 1) / NTHREADS;
+    float v[NIT][4];
+    long long col0[NIT];  // image column of the chunk's first element; a huge value marks "nothing to place"
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {  // all loads first
+        const int e = threadIdx.x + it * NTHREADS;
+        const int ly = e / CH, k = e - ly * CH;
+        const int yy = y0 + ly - S::R;
+        col0[it] = (long long)1 << 40;
+        v[it][0] = v[it][1] = v[it][2] = v[it][3] = 0.f;
+        if (e >= S::XH * CH || yy < 0 || yy >= H || xa >= xb) continue;
+        const size_t row0 = plane0 + (size_t)yy * W;               // tensor-wide index of the row's first element
+        const size_t c = ((row0 + xa) >> 2) + k;                    // aligned chunk
+        if (4 * c >= row0 + xb) continue;
+        if (4 * c + 3 < total) {
+            const float4 t = load_vec4(base + 4 * c);
+            v[it][0] = t.x; v[it][1] = t.y; v[it][2] = t.z; v[it][3] = t.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[it][i] = 4 * c + i < total ? ldf(base + 4 * c + i) : 0.f;
+        }
+        col0[it] = (long long)(4 * c) - (long long)row0;
+    }
+#pragma unroll
+    for (int it = 0; it < NIT; ++it) {
+        const int ly = (threadIdx.x + it * NTHREADS) / CH;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const long long col = col0[it] + i;
+            if (col >= xa && col < xb) Xs[ly][(int)col - x0 + S::R] = v[it][i];
+        }
+    }
+}
+
+template <typename T, int K>
+__device__ __forceinline__ void stage_pixels_looped(const T *__restrict__ base, size_t p, size_t total, int H, int W, int y0,
+                                             int x0, float (*Xs)[SynthTile<K>::XP]) {
+    using S = SynthTile<K>;
+    const size_t plane0 = p * (size_t)H * W;
+    const T *xp = base + plane0;
+    if ((W & 3) == 0) {
+        for (int e = threadIdx.x; e < S::XH * (STW / 4); e += NTHREADS) {
+            const int ly = e / (STW / 4), j = e - ly * (STW / 4);
+            const int yy = y0 + ly - S::R, xx = x0 + 4 * j;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (yy >= 0 && yy < H && xx < W) v = load_vec4(xp + (size_t)yy * W + xx);
+            float *q = &Xs[ly][S::R + 4 * j];
+            q[0] = v.x; q[1] = v.y; q[2] = v.z; q[3] = v.w;
+        }
+        for (int e = threadIdx.x; e < S::XH * (S::XP - STW); e += NTHREADS) {
+            const int ly = e / (S::XP - STW), h = e - ly * (S::XP - STW);
+            const int lx = h < S::R ? h : STW + h;  // left halo, then right halo and the pitch padding
+            const int yy = y0 + ly - S::R, xx = x0 + lx - S::R;
+            Xs[ly][lx] = (yy >= 0 && yy < H && xx >= 0 && xx < W) ? ldf(xp + (size_t)yy * W + xx) : 0.f;
+        }
+        return;
+    }
+    float4 *z = reinterpret_cast<float4 *>(&Xs[0][0]);
+    for (int e = threadIdx.x; e < S::XH * S::XP / 4; e += NTHREADS) z[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+    constexpr int CH = (S::XW + 3) / 4 + 1;  // aligned chunks that can overlap one tile row
+    const int xa = x0 - S::R < 0 ? 0 : x0 - S::R;                    // first image column the tile needs
+    const int xb = x0 + STW + S::R > W ? W : x0 + STW + S::R;        // one past the last
     for (int e = threadIdx.x; e < S::XH * CH; e += NTHREADS) {
         const int ly = e / CH, k = e - ly * CH;
         const int yy = y0 + ly - S::R;
@@ -326,6 +463,13 @@ __device__ __forceinline__ void stage_pixels(const T *__restrict__ base, size_t 
             if (col >= xa && col < xb) Xs[ly][(int)col - x0 + S::R] = v[i];
         }
     }
+}
+
+template <typename T, int K, bool BATCH>
+__device__ __forceinline__ void stage_pixels(const T *__restrict__ base, size_t p, size_t total, int H, int W, int y0,
+                                             int x0, float (*Xs)[SynthTile<K>::XP]) {
+    if (BATCH) stage_pixels_batched<T, K>(base, p, total, H, W, y0, x0, Xs);
+    else stage_pixels_looped<T, K>(base, p, total, H, W, y0, x0, Xs);
 }
 
 // Proposition 2 for the 4 x 4 pixel block with origin (Y0, X0), both multiples of 4, of plane p: level 1
@@ -452,7 +596,7 @@ synth_fwd_kernel(const T *__restrict__ x, int H, int W, int C, int L, const floa
     const int ntx = tiles_of(W, STW), ntile = ntx * tiles_of(H, STH);
     const int p = blockIdx.x / ntile, tile = blockIdx.x - p * ntile, c = p % C;
     const int x0 = (tile % ntx) * STW, y0 = (tile / ntx) * STH;
-    stage_pixels<T, K>(x, (size_t)p, (size_t)(gridDim.x / ntile) * H * W, H, W, y0, x0, Xs);
+    stage_pixels<T, K, true>(x, (size_t)p, (size_t)(gridDim.x / ntile) * H * W, H, W, y0, x0, Xs);
     // folded weights (Eq. 8) go through shared memory once, then live in registers
     __shared__ float Ws[K * K + 1];
     const float sc = __ldg(s0 + c);
@@ -532,8 +676,9 @@ level_bwd_kernel(const Tin *__restrict__ Xprev, const Tin *__restrict__ Gprev, i
     for (int b = part; b < B; b += bsplit) {
         const size_t p = (size_t)b * C + c;
         __syncthreads();
-        stage_subbands<Tin, K>(Xprev + p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
-        stage_subbands<Tin, K>(Gprev + p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ds);
+        // (three resident blocks at k <= 5 leave 80 registers: no room for batched loads)
+        stage_subbands<Tin, K, (K > 5)>(Xprev + p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ys);
+        stage_subbands<Tin, K, (K > 5)>(Gprev + p * Hp * Wp, Hp, Wp, Hl, Wl, i0, j0, Ds);
         __syncthreads();
         if (!live) continue;
         // weight gradient: the block's 16 D values (zero outside the grid) against the shifted Y window
@@ -609,8 +754,8 @@ synth_bwd_kernel(const T *__restrict__ x, const T *__restrict__ g, int H, int W,
     for (int b = part; b < B; b += bsplit) {
         const size_t p = (size_t)b * C + c;
         __syncthreads();
-        stage_pixels<T, K>(x, p, (size_t)B * C * H * W, H, W, y0, x0, Xs);
-        stage_pixels<T, K>(g, p, (size_t)B * C * H * W, H, W, y0, x0, Gs);
+        stage_pixels<T, K, (K > 5)>(x, p, (size_t)B * C * H * W, H, W, y0, x0, Xs);
+        stage_pixels<T, K, (K > 5)>(g, p, (size_t)B * C * H * W, H, W, y0, x0, Gs);
         __syncthreads();
         if (!live) continue;
         // weight gradient: the block's 16 upstream values (zero outside the image) against the shifted x window
