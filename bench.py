@@ -1,24 +1,30 @@
 #!/usr/bin/env python
 """Benchmark of the WTConv hot path (forward + backward) on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME] [--no-table]
 
-One "step" = wtconv_forward + wtconv_backward over one batch of the workload (default: the
-WTConvNeXt-T stage-1 block shape in fp32, B=64 C=96 56x56 k=5 L=3).  Prints ONE JSON line.
+Headline workload (default): the full WTConvNeXt-T stage set in bf16 storage / fp32 arithmetic at B = 128
+per GPU, k = 5: (C=96, 56x56, L=3), (C=192, 28x28, L=2), (C=384, 14x14, L=1), (C=768, 7x7, L=1).  One
+"step" = wtconv_forward + wtconv_backward on each of the four stage tensors.  Prints ONE JSON line.
 
-  value        elements/s (N = B*C*H*W per step and rank, summed over ranks), inputs resident in HBM
-  e2e          the same metric through wtconv_step_host: pinned HOST buffers, H2D and D2H copies inside
-  roofline     the dominant kernel (the whole-plane forward / input-gradient kernel) against the FP32
-               ALU roof, from CUDA events around the forward call inside the timed steps
-  cpu_baseline the fp64 oracle on this machine's host cores (rank 0, N=1 only)
+  value          elements/s: sum of the stages' B*C*H*W per step (times the ranks) / step time, inputs in HBM
+  ms_per_step    median over repeated regions of exactly K steps (regions repeat until >= 0.5 s is timed)
+  e2e            the same metric through wtconv_step_host: pinned HOST buffers, H2D and D2H copies inside
+  roofline       the dominant kernel of the stage that sits furthest below its roof, against the FP32 ALU roof
+  per_workload   every benchmark configuration (level sweep fp32/fp16, stage-1 fp32, the stage set, the
+                 network's depth schedule, k = 3 / 7, the large planes) with forward / backward time,
+                 elements/s, ALU and HBM fractions and the kernel family that served it (N = 1 only)
+  cpu_baseline   the fp64 oracle on this machine's host cores on a bounded sample (rank 0, N = 1 only)
 
-Under torchrun (N > 1) every rank runs the same per-rank batch (weak scaling); the parameter
-gradients are summed across ranks with one NCCL all-reduce per step (the only exchange the
-batch-sharded operator has).  `--impl reference` times the CPU oracle instead (rank 0 only).
+`--workload NAME` times that single workload instead of the stage set (used for profiler captures).
+Under torchrun (N > 1) every rank runs the same per-rank batch (weak scaling); the parameter gradients of
+a stage live in one flat buffer that is summed across ranks with one NCCL all-reduce per stage and step.
+`--impl reference` times the CPU oracle instead (rank 0 only).
 """
 import argparse
 import json
 import os
+import statistics
 import subprocess
 import sys
 import threading
@@ -28,13 +34,22 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FP32 lanes x 2 FLOP x max SM clock = 74.4
+PEAK_SOURCE = "derived: 148 SMs x 128 FP32 lanes x 2 FLOP x 1.965 GHz (a packed-FMA loop measured 74.1 on this pool)"
+L2_BYTES = 126 << 20
+
+STAGE_SET = ["stage1_bf16", "stage2_bf16", "stage3_bf16", "stage4_bf16"]
+TABLE = (["stage1_f32"] + ["sweep_L%d_f32" % l for l in range(1, 6)] + ["sweep_L%d_f16" % l for l in range(1, 6)] +
+         STAGE_SET + ["convnext_s%d_bf16" % s for s in range(1, 5)] + ["stage1_k3_f32", "stage1_k7_f32"] +
+         ["large_f16", "large_odd_f16"])
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (bytes; keyed by workload and kernel).  None where no capture exists.
-NCU_DRAM_TRAFFIC = {
-    ("stage1_f32", "plane_bwd_kernel"): 154664704 + 48539904,
-    ("stage1_f32", "plane_fwd_kernel"): 77319680 + 32544768,
-}
+# (bytes; keyed by workload and kernel family).  Absent = no capture of that launch exists.
+NCU_DRAM_TRAFFIC = {}
+try:
+    with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as _f:
+        NCU_DRAM_TRAFFIC = {tuple(k.split("|")): v for k, v in json.load(_f).items() if not k.startswith("_")}
+except Exception:
+    pass
 
 
 def load_measured_peaks():
@@ -96,62 +111,176 @@ class ClockSampler:
                 "samples": len(mhz), "power_w_max": max(pw) if pw else None}
 
 
-def run_reference(args, wl):
-    """The CPU oracle, as it stands, on this box's host cores (bounded sample of the workload)."""
-    import numpy as np
+def oracle_step_seconds(wls, reps):
+    """Seconds per fwd+bwd of the fp64 oracle over the given (batch-reduced) workloads; returns (s, elements)."""
     from oracle import wtconv_oracle as O
     from paper_2608_10805_b200 import inputs
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    Bs = min(wl.B, args.ref_batch)
-    wls = wl.with_(B=Bs)
-    I = inputs.make_inputs(wls)
-    step = lambda: (O.forward(I["x"], I["w0"], I["s0"], None, I["wl"], I["sl"], wls.L),
-                    O.backward(I["x"], I["g"], I["w0"], I["s0"], None, I["wl"], I["sl"], wls.L))
-    for _ in range(args.warmup):
-        step()
+    Is = [inputs.make_inputs(w) for w in wls]
+    def step():
+        for w, I in zip(wls, Is):
+            O.forward(I["x"], I["w0"], I["s0"], None, I["wl"], I["sl"], w.L)
+            O.backward(I["x"], I["g"], I["w0"], I["s0"], None, I["wl"], I["sl"], w.L)
+    step()
     t0 = time.time()
-    for _ in range(args.steps):
+    for _ in range(reps):
         step()
-    dt = time.time() - t0
-    val = wls.N * args.steps / dt
-    sample = "fwd+bwd of B=%d of %d images of %s (per-plane cost is batch-independent)" % (Bs, wl.B, wl.name)
+    return (time.time() - t0) / reps, sum(w.N for w in wls)
+
+
+def run_reference(args, wls, name):
+    """The CPU oracle, as it stands, on this box's host cores (bounded sample of the workload)."""
+    from oracle import wtconv_oracle as O
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    Bs = min(min(w.B for w in wls), args.ref_batch)
+    sample_wls = [w.with_(B=Bs) for w in wls]
+    steps = max(1, min(args.steps, 5))
+    dt, n = oracle_step_seconds(sample_wls, steps)
+    val = n / dt
+    sample = "fwd+bwd of B=%d of %d images of %s (per-plane cost is batch-independent)" % (Bs, wls[0].B, name)
     print(json.dumps({
         "impl": "reference", "metric": "wtconv_fwd_bwd_elements_per_s", "value": val, "unit": "elements/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "n_gpus": args.gpus, "steps": steps, "warmup": 1, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "B": wl.B, "C": wl.C, "H": wl.H, "W": wl.W, "k": wl.k, "L": wl.L,
-                   "sample_B": Bs},
+        "config": {"workload": name, "stages": [w.name for w in wls], "sample_B": Bs},
         "cpu_baseline": {"value": val, "unit": "elements/s", "cores": O.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
 
+class Runner:
+    """Device buffers of one workload and the two library calls of a step."""
+
+    def __init__(self, wl, dev, rank, tune, torch, wt, inputs, dp):
+        self.wl, self.torch, self.wt = wl, torch, wt
+        tdt = wt.DTYPE_NAMES[wl.dtype]
+        self.esz = 4 if wl.dtype == "f32" else 2
+        self.desc = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, tdt, tune)
+        # rotating input sets: together with the outputs a pass over all sets touches more than the L2 holds
+        step_bytes = 4 * wl.N * self.esz
+        self.nbuf = 1 if step_bytes > 2 * L2_BYTES else min(8, -(-2 * L2_BYTES // step_bytes) + 1)
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1000 * wl.seed + 17 * rank + 1)
+        shape = (wl.B, wl.C, wl.H, wl.W)
+        self.xs = [torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(tdt) for _ in range(self.nbuf)]
+        self.gs = [torch.randn(shape, generator=gen, device=dev, dtype=torch.float32).to(tdt) for _ in range(self.nbuf)]
+        P = inputs.make_inputs(wl.with_(B=1))  # parameters do not depend on B (own Philox stream per tensor)
+        up = lambda a: torch.from_numpy(a).to(dev).contiguous()
+        self.w0, self.s0, self.wl_, self.sl = up(P["w0"]), up(P["s0"]), up(P["wl"]), up(P["sl"])
+        self.out, self.gx = torch.empty_like(self.xs[0]), torch.empty_like(self.xs[0])
+        self.grads = dp.FlatGrads(wl.C, wl.k, wl.L, bias=False, device=dev)
+        self.ws = wt.alloc_workspace(self.desc, dev)
+        self.ws_fwd, self.ws_bwd = wt.wtconv_workspace_bytes(self.desc)
+        self.nf, self.nb = wt.wtconv_launch_count(self.desc)
+        self.plan = wt.wtconv_plan_name(self.desc)
+
+    def fwd(self, i, stream):
+        self.wt.wtconv_forward(self.desc, self.xs[i % self.nbuf], self.w0, self.s0, None, self.wl_, self.sl, self.out,
+                               self.ws, stream)
+
+    def bwd(self, i, stream):
+        g = self.grads
+        self.wt.wtconv_backward(self.desc, self.xs[i % self.nbuf], self.gs[i % self.nbuf], self.w0, self.s0, None,
+                                self.wl_, self.sl, self.gx, g["dw0"], g["ds0"], None, g["dwl"], g["dsl"], self.ws, stream)
+
+    def device_bytes(self):
+        act = self.wl.N * self.esz
+        par = 4 * sum(t.numel() for t in (self.w0, self.s0, self.wl_, self.sl))
+        return {"x": act, "out": act, "params": par, "workspace_fwd": self.ws_fwd, "workspace_bwd": self.ws_bwd,
+                "forward_peak": 2 * act + par + self.ws_fwd,
+                "training_step_peak": 4 * act + 2 * par + max(self.ws_fwd, self.ws_bwd)}
+
+
+def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions):
+    """Regions of exactly K steps, repeated until `min_seconds` have been timed; every call is bracketed by events.
+    Returns (region_ms list, per-runner [fwd_ms list, bwd_ms list])."""
+    def step(i, ev=None):
+        for j, r in enumerate(runners):
+            if ev is not None:
+                ev[j][0].record(stream)
+            r.fwd(i, stream)
+            if ev is not None:
+                ev[j][1].record(stream)
+            r.bwd(i, stream)
+            if ev is not None:
+                ev[j][2].record(stream)
+            all_reduce(r)
+    for i in range(warmup):
+        step(i)
+    sync_all()
+    regions, fwd, bwd = [], [[] for _ in runners], [[] for _ in runners]
+    total = 0.0
+    while len(regions) < max_regions and (total < min_seconds or not regions):
+        evs = [[tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in runners] for _ in range(K)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sync_all()
+        e0.record(stream)
+        for i in range(K):
+            step(i, evs[i])
+        e1.record(stream)
+        sync_all()
+        ms = e0.elapsed_time(e1)
+        regions.append(ms)
+        total += ms * 1e-3
+        for ev in evs:
+            for j in range(len(runners)):
+                fwd[j].append(ev[j][0].elapsed_time(ev[j][1]))
+                bwd[j].append(ev[j][1].elapsed_time(ev[j][2]))
+    return regions, fwd, bwd
+
+
+def row_for(r, fwd_ms, bwd_ms, peaks, io_model):
+    wl = r.wl
+    fl_f = io_model.algorithmic_flops(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, "fwd")
+    by_f = io_model.compulsory_bytes(wl.N, r.esz, "fwd")
+    by_s = io_model.compulsory_bytes(wl.N, r.esz, "fwd+bwd")
+    peak_f, peak_b = FP32_ALU_PEAK_TFLOPS * 1e12, peaks["hbm_gbs"] * 1e9
+    t_f, t_b = fwd_ms * 1e-3, bwd_ms * 1e-3
+    t_s = t_f + t_b
+    alu_floor, hbm_floor = 3 * fl_f / peak_f, by_s / peak_b
+    return {
+        "workload": wl.name, "shape": [wl.B, wl.C, wl.H, wl.W], "k": wl.k, "L": wl.L, "storage": wl.dtype,
+        "plan": r.plan, "launches": [r.nf, r.nb],
+        "fwd_us": round(fwd_ms * 1e3, 2), "bwd_us": round(bwd_ms * 1e3, 2),
+        "fwd_gelem_s": round(wl.N / t_f / 1e9, 2), "gelem_s": round(wl.N / t_s / 1e9, 2),
+        "fwd_alu_frac": round(fl_f / t_f / peak_f, 4), "bwd_alu_frac": round(2 * fl_f / t_b / peak_f, 4),
+        "alu_frac": round(3 * fl_f / t_s / peak_f, 4),
+        "fwd_hbm_frac_of_measured": round(by_f / t_f / peak_b, 4), "hbm_frac_of_measured": round(by_s / t_s / peak_b, 4),
+        "bound": "alu" if alu_floor >= hbm_floor else "hbm",
+        "roof_frac": round(max(alu_floor, hbm_floor) / t_s, 4),
+        "workspace_bytes": [r.ws_fwd, r.ws_bwd],
+        "paper_q_fused_fwd_N": round(io_model.q_fused(wl.L), 3) if wl.L else None,
+        "paper_q_ref_fwd_N": round(io_model.q_ref(wl.L), 3) if wl.L else None,
+    }
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="stage1_f32")
+    ap.add_argument("--workload", default="stage_set_bf16", help="stage_set_bf16 (default) or one workload name")
     ap.add_argument("--ref-batch", type=int, default=16, help="images per oracle step in --impl reference")
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="repeat the K-step region until this much is timed")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true", help="skip the per_workload table")
+    ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--tune", type=lambda s: int(s, 0), default=0, help="launch-plan override bits (see wtconv.h)")
     args = ap.parse_args()
 
     from paper_2608_10805_b200 import inputs, io_model
-    wl = inputs.WORKLOADS[args.workload]
+    names = STAGE_SET if args.workload == "stage_set_bf16" else [args.workload]
+    wls = [inputs.WORKLOADS[n] for n in names]
+    head_name = "wtconvnext_t_stage_set_bf16_B128" if args.workload == "stage_set_bf16" else args.workload
     if args.impl == "reference":
-        args.steps = min(args.steps, 5)
-        args.warmup = min(args.warmup, 1)
-        return run_reference(args, wl)
+        return run_reference(args, wls, head_name)
 
-    import numpy as np
     import torch
     import torch.distributed as dist
+    from paper_2608_10805_b200 import dp
     from paper_2608_10805_b200 import wtconv as wt
 
     rank = int(os.environ.get("RANK", "0"))
@@ -165,98 +294,74 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=dev)
     wt.lib()  # fail loudly here if the CUDA library is missing
-
-    tdt = wt.DTYPE_NAMES[wl.dtype]
-    esz = 4 if wl.dtype == "f32" else 2
-    desc = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, tdt, args.tune)
-    # seeded synthetic inputs (per-rank stream), two rotating input sets so no step re-reads a warm L2
-    nbuf = 2
-    sets = []
-    for i in range(nbuf):
-        I = inputs.make_inputs(wl.with_(seed=wl.seed + 100 * rank + 7 * i))
-        sets.append(I)
-    up = lambda a, dt=torch.float32: torch.from_numpy(a).to(dev).to(dt).contiguous()
-    xs = [up(I["x"], tdt) for I in sets]
-    gs = [up(I["g"], tdt) for I in sets]
-    P = sets[0]
-    w0, s0, wl_, sl = up(P["w0"]), up(P["s0"]), up(P["wl"]), up(P["sl"])
-    out, gx = torch.empty_like(xs[0]), torch.empty_like(xs[0])
-    gw0, gs0, gwl, gsl = torch.empty_like(w0), torch.empty_like(s0), torch.empty_like(wl_), torch.empty_like(sl)
-    flat_grads = [gw0, gs0, gwl, gsl]
-    ws = wt.alloc_workspace(desc, dev)
     stream = torch.cuda.current_stream()
-
-    def step(i, ev=None):
-        x, g = xs[i % nbuf], gs[i % nbuf]
-        if ev:
-            ev[0].record(stream)
-        wt.wtconv_forward(desc, x, w0, s0, None, wl_, sl, out, ws, stream)
-        if ev:
-            ev[1].record(stream)
-        wt.wtconv_backward(desc, x, g, w0, s0, None, wl_, sl, gx, gw0, gs0, None, gwl, gsl, ws, stream)
-        if ev:
-            ev[2].record(stream)
-        if world > 1:
-            for t in flat_grads:
-                dist.all_reduce(t)
 
     def sync_all():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    # keep the GPU busy for a moment so the sampled clocks are the clocks under load
-    sync_all()
+    def all_reduce(r):
+        if world > 1:
+            r.grads.all_reduce()  # one collective per stage and step: the flat parameter-gradient buffer
+
+    mk = lambda w, tune=0: Runner(w, dev, rank, tune, torch, wt, inputs, dp)
+    runners = [mk(w, args.tune) for w in wls]
+    K, W = max(args.steps, 1), max(args.warmup, 3)
+    for i in range(3):  # first calls: plan search, function attributes, module load
+        for r in runners:
+            r.fwd(i, stream); r.bwd(i, stream)
     sync_all()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-        time.sleep(0.3)
-    K = args.steps
-    fev = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in range(K)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync_all()
+        time.sleep(0.2)
     t0 = time.time()
-    e0.record(stream)
-    for i in range(K):
-        step(i, fev[i])
-    e1.record(stream)
-    sync_all()
+    regions, fwd_ms, bwd_ms = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400)
     t1 = time.time()
-    ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
+    med = statistics.median(regions)
+    ms = torch.tensor([med], device=dev)
     if world > 1:
         dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_total = float(ms.item())
+    ms_region = float(ms.item())
     clocks = sampler.stop(t0, t1) if rank == 0 else None
-    fwd_kernel_ms = sum(a.elapsed_time(b) for a, b, _ in fev) / len(fev)
-    bwd_call_ms = sum(b.elapsed_time(c) for _, b, c in fev) / len(fev)
 
     # ---- end to end through the host entry point: pinned host buffers, copies inside the timed region
-    hb = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory()
-    hx, hg = xs[0].cpu().pin_memory(), gs[0].cpu().pin_memory()
-    hw0, hs0, hwl, hsl = (t.cpu().pin_memory() for t in (w0, s0, wl_, sl))
-    hout, hgx, hgw0, hgs0, hgwl, hgsl = hb(out), hb(gx), hb(gw0), hb(gs0), hb(gwl), hb(gsl)
-    hws = torch.empty(wt.wtconv_step_host_workspace_bytes(desc), dtype=torch.uint8, device=dev)
+    e2e = None
+    if not args.no_e2e:
+        host = []
+        for r in runners:
+            hb = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory()
+            g = r.grads
+            host.append(dict(
+                hx=r.xs[0].cpu().pin_memory(), hg=r.gs[0].cpu().pin_memory(),
+                hp=[t.cpu().pin_memory() for t in (r.w0, r.s0, r.wl_, r.sl)],
+                ho=[hb(r.out), hb(r.gx), hb(g["dw0"]), hb(g["ds0"]), hb(g["dwl"]), hb(g["dsl"])],
+                ws=torch.empty(wt.wtconv_step_host_workspace_bytes(r.desc), dtype=torch.uint8, device=dev)))
 
-    def host_step():
-        wt.wtconv_step_host(desc, hx, hg, hw0, hs0, None, hwl, hsl, hout, hgx, hgw0, hgs0, None, hgwl, hgsl, hws, stream)
-    host_step()
-    sync_all()
-    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    h0.record(stream)
-    for _ in range(args.e2e_steps):
+        def host_step():
+            for r, h in zip(runners, host):
+                wt.wtconv_step_host(r.desc, h["hx"], h["hg"], h["hp"][0], h["hp"][1], None, h["hp"][2], h["hp"][3],
+                                    h["ho"][0], h["ho"][1], h["ho"][2], h["ho"][3], None, h["ho"][4], h["ho"][5],
+                                    h["ws"], stream)
         host_step()
-    h1.record(stream)
-    sync_all()
-    hms = torch.tensor([h0.elapsed_time(h1)], device=dev)
-    if world > 1:
-        dist.all_reduce(hms, op=dist.ReduceOp.MAX)
-    e2e_val = wl.N * world * args.e2e_steps / (float(hms.item()) * 1e-3)
-    psz = sum(t.numel() * 4 for t in (w0, s0, wl_, sl))
-    h2d = 2 * wl.N * esz + psz
-    d2h = 2 * wl.N * esz + psz
+        sync_all()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(args.e2e_steps):
+            host_step()
+        h1.record(stream)
+        sync_all()
+        hms = torch.tensor([h0.elapsed_time(h1)], device=dev)
+        if world > 1:
+            dist.all_reduce(hms, op=dist.ReduceOp.MAX)
+        n_step = sum(r.wl.N for r in runners)
+        psz = sum(4 * sum(t.numel() for t in (r.w0, r.s0, r.wl_, r.sl)) for r in runners)
+        act = sum(2 * r.wl.N * r.esz for r in runners)
+        e2e = {"value": n_step * world * args.e2e_steps / (float(hms.item()) * 1e-3), "unit": "elements/s",
+               "h2d_bytes_per_step": act + psz, "d2h_bytes_per_step": act + psz, "steps": args.e2e_steps,
+               "api": "wtconv_step_host (host pointers; uploads, kernels and downloads pipelined by batch chunk)"}
+        del host
 
     if rank != 0:
         if world > 1:
@@ -264,67 +369,80 @@ def main():
         return
 
     peaks, peak_kind = load_measured_peaks()
-    ms_step = ms_total / K
-    value = wl.N * world * K / (ms_total * 1e-3)
-    fl_fwd = io_model.algorithmic_flops(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, "fwd")
-    fl_bwd = io_model.algorithmic_flops(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, "bwd")
-    fl_step = io_model.algorithmic_flops(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, "fwd+bwd")
-    nf, nb = wt.wtconv_launch_count(desc)
-    plane = wt.wtconv_plan_name(desc) == "plane"
-    fused_bwd = plane and nb == 2
-    # dominant kernel: the fused backward kernel (about two thirds of a step) where the plan has one, timed by the
-    # events around wtconv_backward (which also cover its small epilogue launch and memset: a conservative rate);
-    # otherwise the forward kernel, timed by the events around wtconv_forward
-    if fused_bwd:
-        dom_name, dom_ms, dom_fl = "plane_bwd_kernel (+ epilogue)", bwd_call_ms, fl_bwd
+    ms_step = ms_region / K
+    n_step = sum(r.wl.N for r in runners)
+    value = n_step * world / (ms_step * 1e-3)
+    mean = lambda v: sum(v) / len(v)
+    rows = [row_for(r, statistics.median(f), statistics.median(b), peaks, io_model) for r, f, b in zip(runners, fwd_ms, bwd_ms)]
+    fl_step = sum(io_model.algorithmic_flops(r.wl.B, r.wl.C, r.wl.H, r.wl.W, r.wl.k, r.wl.L, "fwd+bwd") for r in runners)
+    by_step = sum(io_model.compulsory_bytes(r.wl.N, r.esz, "fwd+bwd") for r in runners)
+    alu_floor_ms = fl_step / (FP32_ALU_PEAK_TFLOPS * 1e12) * 1e3
+    hbm_floor_ms = by_step / (peaks["hbm_gbs"] * 1e9) * 1e3
+    # roofline: the stage furthest below its roof, and of its two calls the longer one
+    worst = min(range(len(rows)), key=lambda j: rows[j]["roof_frac"])
+    wr, wrow = runners[worst], rows[worst]
+    fl_f = io_model.algorithmic_flops(wr.wl.B, wr.wl.C, wr.wl.H, wr.wl.W, wr.wl.k, wr.wl.L, "fwd")
+    if wrow["bwd_us"] >= wrow["fwd_us"]:
+        dom_kind, dom_ms, dom_fl = "backward", mean(bwd_ms[worst]), 2 * fl_f
     else:
-        dom_name, dom_ms, dom_fl = ("plane_fwd_kernel" if plane else "tiled forward launches"), fwd_kernel_ms, fl_fwd
+        dom_kind, dom_ms, dom_fl = "forward", mean(fwd_ms[worst]), fl_f
     achieved = dom_fl / (dom_ms * 1e-3) / 1e12
-    hbm_step = io_model.compulsory_bytes(wl.N, esz, "fwd+bwd")
     result = {
         "metric": "wtconv_fwd_bwd_elements_per_s", "value": value, "unit": "elements/s", "n_gpus": world,
-        "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "B_per_gpu": wl.B, "C": wl.C, "H": wl.H, "W": wl.W, "k": wl.k, "L": wl.L,
-                   "storage_dtype": wl.dtype, "plan": wt.wtconv_plan_name(desc),
-                   "l2": "two rotating input sets; a step touches %d MB > 126 MB L2" % (4 * wl.N * esz // 2 ** 20),
-                   "parallelism": "dp%d (batch-sharded, NCCL all-reduce of parameter gradients)" % world},
+        "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wt.ARITHMETIC_DTYPE, "data": "synthetic",
+        "config": {"workload": head_name,
+                   "stages": [{"name": r.wl.name, "B_per_gpu": r.wl.B, "C": r.wl.C, "H": r.wl.H, "W": r.wl.W, "k": r.wl.k,
+                               "L": r.wl.L, "storage_dtype": r.wl.dtype, "plan": r.plan} for r in runners],
+                   "l2": "a step touches %d MB (> 126 MB L2) over rotating input sets" %
+                         (sum(4 * r.wl.N * r.esz * (r.nbuf if len(runners) == 1 else 1) for r in runners) >> 20),
+                   "timing": "median of %d regions of %d steps (%.2f s timed); CUDA events on the launch stream"
+                             % (len(regions), K, sum(regions) * 1e-3),
+                   "parallelism": "dp%d (batch-sharded; one all-reduce of the flat parameter-gradient buffer per stage)" % world},
         "clocks": clocks,
-        "e2e": {"value": e2e_val, "unit": "elements/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": args.e2e_steps},
-        "gpu_launches": (nf + nb) * K,
-        "roofline": {"bound": "alu", "kernel": dom_name,
+        "ms_per_step_x_sm_mhz": ms_step * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,
+        "region_ms": {"min": min(regions), "median": med, "max": max(regions), "n": len(regions)},
+        "e2e": e2e,
+        "gpu_launches": sum(r.nf + r.nb for r in runners) * K,
+        "roofline": {"bound": wrow["bound"], "kernel": "%s call of %s (%s kernels)" % (dom_kind, wr.wl.name, wr.plan),
                      "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
-                     "frac": achieved / FP32_ALU_PEAK_TFLOPS, "traffic": NCU_DRAM_TRAFFIC.get((wl.name, dom_name.split()[0])),
-                     "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 FLOP x 1.965 GHz (measured 74.1 with a packed-FMA loop)",
-                     "launch_ms": dom_ms, "flops_per_launch": dom_fl,
-                     "forward_kernel": {"launch_ms": fwd_kernel_ms, "achieved": fl_fwd / (fwd_kernel_ms * 1e-3) / 1e12,
-                                        "frac": fl_fwd / (fwd_kernel_ms * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS,
-                                        "traffic": NCU_DRAM_TRAFFIC.get((wl.name, "plane_fwd_kernel"))}},
+                     "frac": achieved / FP32_ALU_PEAK_TFLOPS,
+                     "traffic": NCU_DRAM_TRAFFIC.get((wr.wl.name, dom_kind)),
+                     "peak_source": PEAK_SOURCE, "launch_ms": dom_ms, "flops_per_launch": dom_fl},
         "step_rooflines": {
-            "alu_frac": fl_step / (ms_step * 1e-3) / 1e12 / FP32_ALU_PEAK_TFLOPS,
-            "hbm_compulsory_gbs": hbm_step / (ms_step * 1e-3) / 1e9,
-            "hbm_frac_of_%s" % peak_kind: hbm_step / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-            "hbm_frac_of_8TBs": hbm_step / (ms_step * 1e-3) / 1e9 / 8000.0,
-            "alu_floor_ms": fl_step / (FP32_ALU_PEAK_TFLOPS * 1e12) * 1e3,
-            "hbm_floor_ms": hbm_step / (peaks["hbm_gbs"] * 1e9) * 1e3},
-        "paper_io_model": {"q_fused_fwd_N": io_model.q_fused(wl.L), "q_ref_fwd_N": io_model.q_ref(wl.L),
-                           "ours_fwd_N": 2.0, "ours_bwd_N": 3.0 if nb == 2 else 4.0},
+            "alu_frac": alu_floor_ms / ms_step,
+            "hbm_compulsory_gbs": by_step / (ms_step * 1e-3) / 1e9,
+            "hbm_frac_of_%s" % peak_kind: hbm_floor_ms / ms_step,
+            "hbm_frac_of_8TBs": by_step / (ms_step * 1e-3) / 1e9 / 8000.0,
+            "alu_floor_ms": alu_floor_ms, "hbm_floor_ms": hbm_floor_ms,
+            "roof_frac": max(alu_floor_ms, hbm_floor_ms) / ms_step},
+        "device_bytes": {r.wl.name: r.device_bytes() for r in runners},
+        "stages": rows,
     }
     if world == 1 and not args.no_cpu_baseline:
         from oracle import wtconv_oracle as O
-        Bs = min(wl.B, 64)
-        Ic = inputs.make_inputs(wl.with_(B=Bs))
-        reps = 3
-        c0 = time.time()
-        for _ in range(reps):
-            O.forward(Ic["x"], Ic["w0"], Ic["s0"], None, Ic["wl"], Ic["sl"], wl.L)
-            O.backward(Ic["x"], Ic["g"], Ic["w0"], Ic["s0"], None, Ic["wl"], Ic["sl"], wl.L)
-        cdt = (time.time() - c0) / reps
-        result["cpu_baseline"] = {"value": wl.with_(B=Bs).N / cdt, "unit": "elements/s", "cores": O.num_threads(),
+        Bs = min(min(w.B for w in wls), 32)
+        cdt, cn = oracle_step_seconds([w.with_(B=Bs) for w in wls], 3)
+        result["cpu_baseline"] = {"value": cn / cdt, "unit": "elements/s", "cores": O.num_threads(),
                                   "kind": "oracle", "seconds_per_step": cdt,
-                                  "sample": "%d x fwd+bwd of B=%d images of %s, fp64 (%.0f core-seconds)"
-                                            % (reps, Bs, wl.name, reps * cdt * O.num_threads())}
+                                  "sample": "3 x fwd+bwd of B=%d images of %s, fp64 (%.0f core-seconds)"
+                                            % (Bs, head_name, 3 * cdt * O.num_threads())}
+    if world == 1 and not args.no_table:
+        table = []
+        have = {r.wl.name: row for r, row in zip(runners, rows)}
+        del runners
+        torch.cuda.empty_cache()
+        for name in TABLE:
+            if name in have:
+                table.append(have[name])
+                continue
+            r = mk(inputs.WORKLOADS[name])
+            k = 3 if r.wl.N > (1 << 27) else 10
+            _, f, b = time_regions([r], k, 3, stream, torch, sync_all, lambda _r: None, 0.05, 20)
+            table.append(row_for(r, statistics.median(f[0]), statistics.median(b[0]), peaks, io_model))
+            del r
+            torch.cuda.empty_cache()
+        result["per_workload"] = table
     print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()

@@ -72,6 +72,10 @@ typedef enum {
 
 /* desc->flags */
 #define WTCONV_FLAG_TILED_ONLY 1u /* never take the plane-resident kernels (used to test the tiled path) */
+/* Test aid for the timeout path of the bounded device-side waits: no bulk copy is issued at all and the wait
+ * limit is tiny, so every wait for a copy runs out; the kernels record it in the status word and return
+ * normally with nothing in flight (outputs are then invalid by design).  Never set it in production. */
+#define WTCONV_FLAG_TEST_NO_COPY 2u
 /* Launch-plan overrides for the plane-resident kernels, for tuning experiments (0 = let the planner choose):
  *   bits  8-12  threads per block / 32 of the forward / input-gradient kernel
  *   bits 13-15  resident blocks per SM of that kernel
@@ -111,6 +115,10 @@ wtconv_status wtconv_workspace_bytes(const wtconv_desc *desc, size_t *fwd_bytes,
  * kernels, "tiled" = per-level tiled kernels).  Host call; returns NULL for an invalid desc. */
 const char *wtconv_plan_name(const wtconv_desc *desc);
 
+/* Launch plan of a descriptor as text (threads per block, resident blocks per SM, planes per work unit, register
+ * tile rows, prefetch ring depth; "ring=0" = the kernel waits for no copy).  Host call.  Errors: NULL, desc. */
+wtconv_status wtconv_plan_describe(const wtconv_desc *desc, char *buf, size_t n);
+
 /* Number of kernel launches one wtconv_forward / wtconv_backward call enqueues. */
 wtconv_status wtconv_launch_count(const wtconv_desc *desc, int32_t *fwd_launches, int32_t *bwd_launches);
 
@@ -133,7 +141,8 @@ wtconv_status wtconv_backward(const wtconv_desc *desc, const void *x, const void
                               float *grad_wl, float *grad_sl,
                               void *workspace, size_t workspace_bytes, void *stream);
 
-/* Device-side status of the last call that used `workspace` (device pointer) with this descriptor: enqueues on
+/* Device-side status of the last call that used `workspace` (device pointer; NULL = the array built into the
+ * library that wtconv_backward_static uses, on the current device) with this descriptor: enqueues on
  * `stream` a copy of the workspace's status word into *h_flag (a HOST int32, pinned if the copy is to be
  * asynchronous).  Once the stream has reached this point, 0 means every bounded wait inside the kernels
  * completed (the paper's kernels wait for nothing; ours wait only for their own bulk copies); non-zero means a

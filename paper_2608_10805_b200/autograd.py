@@ -6,9 +6,48 @@ on-chip recomputation of Sec. 4.1 applied to training memory).  Parameters are f
 activation dtype.  The layer is Algorithm 1 of the paper: base depthwise conv with scale (and optional
 bias) plus L Haar levels with their own depthwise convs and scales.
 """
+import collections
+
 import torch
 
 from . import wtconv as wt
+
+
+class _StatusWatch:
+    """Deferred check of the kernels' device status word, without synchronising.
+
+    After every library call the status word of its workspace is copied (asynchronously, on the same stream) into
+    a pinned host integer and an event is recorded.  Later calls look at the copies whose events have completed
+    and raise if one is non-zero: a bounded device-side wait ran out in that earlier call and its outputs were not
+    valid.  `drain()` waits for everything outstanding (call it before trusting results at the end of a run)."""
+
+    def __init__(self):
+        self.pending = collections.deque()
+        self.free = []
+
+    def after_call(self, desc, ws):
+        flag = self.free.pop() if self.free else torch.zeros(1, dtype=torch.int32).pin_memory()
+        wt.wtconv_read_status(desc, ws, flag)
+        ev = torch.cuda.Event()
+        ev.record()
+        self.pending.append((ev, flag))
+        self.poll()
+
+    def poll(self, wait=False):
+        while self.pending and (wait or self.pending[0][0].query()):
+            ev, flag = self.pending.popleft()
+            if wait:
+                ev.synchronize()
+            bad = int(flag[0]) != 0
+            self.free.append(flag)
+            if bad:
+                raise wt.WTConvError(11, "a bounded device-side wait ran out in an earlier WTConv call; its outputs are not valid")
+
+    def drain(self):
+        self.poll(wait=True)
+
+
+status_watch = _StatusWatch()
 
 
 class WTConvFunction(torch.autograd.Function):
@@ -27,6 +66,7 @@ class WTConvFunction(torch.autograd.Function):
         out = torch.empty_like(x)
         ws = wt.alloc_workspace(desc, x.device)
         wt.wtconv_forward(desc, x, params[0], params[1], b0c, params[2], params[3], out, ws)
+        status_watch.after_call(desc, ws)
         ctx.desc, ctx.ws, ctx.has_bias = desc, ws, b0 is not None
         ctx.save_for_backward(x, params[0], params[1], b0c if b0c is not None else x.new_empty(0), params[2], params[3])
         return out
@@ -40,6 +80,7 @@ class WTConvFunction(torch.autograd.Function):
         gw0, gs0, gwl, gsl = (torch.empty_like(t) for t in (w0, s0, wl, sl))
         gb0 = torch.empty_like(b0) if b0 is not None else None
         wt.wtconv_backward(ctx.desc, x, g, w0, s0, b0, wl, sl, gx, gw0, gs0, gb0, gwl, gsl, ctx.ws)
+        status_watch.after_call(ctx.desc, ctx.ws)
         return gx, gw0, gs0, gb0, gwl, gsl
 
 

@@ -29,7 +29,9 @@ def build(force=False, verbose=False):
         print(res.stdout)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed building %s" % LIB)
-    with open(os.path.join(HERE, "ptxas_info.txt"), "w") as f:  # registers / spills / shared memory per kernel
+    log_dir = os.path.join(os.path.dirname(HERE), "build")  # registers / spills / shared memory per kernel (not tracked)
+    os.makedirs(log_dir, exist_ok=True)
+    with open(os.path.join(log_dir, "ptxas_info.txt"), "w") as f:
         f.write(res.stdout)
     os.replace(tmp, LIB)
     return LIB

@@ -30,7 +30,9 @@
 //  * Host side: plans (threads, blocks per SM, planes per unit, tile height, ring depth) come from a
 //    search over a small cost model and are cached per shape.
 #pragma once
+#include <atomic>
 #include <cmath>
+#include <cstdio>
 #include <mutex>
 #include <vector>
 #include "common.cuh"
@@ -48,6 +50,7 @@ constexpr int SMEM_PER_SM = 228 * 1024;      // per SM, 1 KB reserved per reside
 constexpr int WT_STRIDE = 28;                // floats per class in the weight table (25 taps, 16-byte padded)
 constexpr int MAX_STAGES = 4;               // deepest prefetch ring (units in flight per block)
 constexpr unsigned WAIT_LIMIT = 1u << 20;    // bounded number of (suspending) waits on the copy barrier: never an endless loop
+constexpr unsigned WAIT_LIMIT_TEST = 64;     // the same under WTCONV_FLAG_TEST_NO_COPY (no copy is ever issued: every wait runs out)
 
 // ------------------------------------------------------------------ bulk-copy (TMA, untiled) helpers
 __device__ __forceinline__ unsigned smem_addr(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -66,10 +69,10 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, unsigned by
                  : "memory");
 }
 // Bounded wait for phase `parity` of `bar`: try_wait suspends the thread for a hardware-limited time per call, so
-// waiting costs few instructions; false if the phase did not complete within WAIT_LIMIT calls.
-__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity) {
+// waiting costs few instructions; false if the phase did not complete within `limit` calls.
+__device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned parity, unsigned limit) {
     const unsigned a = smem_addr(bar);
-    for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
+    for (unsigned i = 0; i < limit; ++i) {
         unsigned ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
                      : "=r"(ok)
@@ -89,15 +92,6 @@ __device__ __forceinline__ void bulk_s2g(void *gdst, const void *src, unsigned b
 __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // order earlier generic-proxy accesses of shared memory before later async-proxy (bulk copy) writes
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-#ifdef WT_PHASE_TIMING
-__device__ unsigned long long wt_phase_cycles[32];
-#define WT_TICK(i) do { if (threadIdx.x == 0 || threadIdx.x == blockDim.x - 1) { long long now_ = clock64(); atomicAdd(&wt_phase_cycles[(i) + (threadIdx.x ? 16 : 0)], (unsigned long long)(now_ - tick_)); tick_ = now_; } } while (0)
-#define WT_TICK_INIT long long tick_ = clock64();
-#else
-#define WT_TICK(i)
-#define WT_TICK_INIT
-#endif
 
 // ------------------------------------------------------------------ geometry (host-planned, passed by value)
 // Division by a launch-invariant divisor as multiply-high: exact while dividend * divisor < 2^32.
@@ -132,6 +126,7 @@ struct Geom {
                                            // weights and gradient accumulators while it walks through the images)
     int nthreads, nblocks, blocks_per_sm;
     int vec;                               // 1: W % 4 == 0, rows are staged with 4-element vector loads
+    int no_copy;                           // test mode: bulk copies are never issued and waits give up quickly (the timeout path)
     int bulk;                              // 1: planes are fetched ahead with cp.async.bulk into a ring of raw buffers at raw_off
     int nstage, stage_bytes;               // ring depth (units in flight) and bytes per ring entry
     int raw_off, raw_slot_bytes, plane_bytes;  // raw staging buffer (float offset), bytes per plane slot / per plane
@@ -142,7 +137,7 @@ struct Geom {
     int npatch;                            // staging work items per plane (vec: 2x4 pixel patches, else 2x2 blocks)
     FastDiv d_npatch, d_prow;              // / npatch, / (patches per patch-row)
     FastDiv d_lvl[MAXL + 1], d_lvlw[MAXL + 1];  // / (Hl*Wl), / Wl   (levels >= 2 staging)
-    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase, d_B;
+    FastDiv d_nlv, d_nt[MAXL + 1], d_tx[MAXL + 1], d_nbase;
     // weight-gradient kernel: class-major thread allocation and partial-sum slots
     int thr_start[4 * MAXL + 2];
     int np;
@@ -566,6 +561,7 @@ __device__ __forceinline__ void issue_unit_copies(unsigned long long *bar, char 
                                                   const T *__restrict__ src, const T *__restrict__ src2, int c0, int b) {
     // the unit (NPL consecutive channels of image b) is one contiguous, 16-byte aligned chunk
     const unsigned bytes = (unsigned)g.NPL * g.plane_bytes;
+    if (g.no_copy) return;  // test mode: the barrier is never armed, nothing is in flight
     mbar_expect_tx(bar, bytes * (src2 ? 2u : 1u));
     const size_t po = ((size_t)b * g.C + c0) * g.H * g.W;
     bulk_g2s(raw, src + po, bytes, bar);
@@ -583,6 +579,20 @@ __device__ __forceinline__ void start_prefetch(unsigned long long *bar, char *ra
     for (int s = 0; s < g.nstage && u_begin + s < u_end; ++s) {
         const int cgs = (u_begin + s) / g.B;
         issue_unit_copies<T>(bar + s, raw + s * g.stage_bytes, g, src, src2, cgs * g.NPL, u_begin + s - cgs * g.B);
+    }
+}
+
+// A bounded wait ran out: the block records it in the status word and stops working (its outputs are invalid
+// anyway).  Before it leaves, every thread waits - again with the limit - for the copies that are still on
+// their way into the ring (the entries of the next nstage - 1 units and the one that was late), so that no
+// copy lands in shared memory the block has already given back.
+__device__ __forceinline__ void give_up_after_timeout(unsigned long long *bar, const Geom &g, int ring, unsigned parity, int u,
+                                                      int u_end, int *status) {
+    if (threadIdx.x == 0) atomicExch(status, 1);
+    const unsigned limit = g.no_copy ? WAIT_LIMIT_TEST : WAIT_LIMIT;
+    for (int s = 0; s < g.nstage && u + s < u_end; ++s) {
+        mbar_wait(bar + ring, parity, limit);
+        if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
     }
 }
 
@@ -777,7 +787,6 @@ __global__ void __launch_bounds__(MAXT, MINB)
 plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0,
                  const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
                  const float *__restrict__ sl, T *__restrict__ out, int *__restrict__ status) {
-    WT_TICK_INIT
     extern __shared__ __align__(16) float sm[];
     const int tid = threadIdx.x, nthr = blockDim.x;
     float *wtab = sm + g.wtab_off;
@@ -789,6 +798,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     zero_fill(sm, g);
     unsigned parity = 0;
     int ring = 0;  // ring entry the current unit arrives in
+    const unsigned wait_limit = g.no_copy ? WAIT_LIMIT_TEST : WAIT_LIMIT;
     const int L = g.L, nlv = g.lvl_start[L + 1];
     const int nlevel_items = g.NPL * nlv, nitems = nlevel_items + g.NPL * g.nbase;
     const size_t HW = (size_t)g.H * g.W;
@@ -818,22 +828,21 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
     PatchD patch1 = decode_patch(g, g.offA, hoist_patch && srank < nstagers ? srank + nstagers : 0x3fffffff);
     __syncthreads();
-    WT_TICK(9);
-    for (int u = u_begin; u < u_end; ++u) {
-        const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
+    // (channel group, image) of the current unit, carried along instead of divided out per unit
+    int cg = u_begin / g.B, b = u_begin - cg * g.B;
+    for (int u = u_begin; u < u_end; ++u, (++b == g.B ? (b = 0, ++cg) : 0)) {
+        const int c = cg * g.NPL;
         const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
-        WT_TICK(0);
         if (c != c_prev) {  // units are group-major: the tables survive all images of a channel group
             build_weight_table(wtab, g, c, FLIP, w0, s0, FLIP ? nullptr : b0, wl, sl);
             c_prev = c;
         }
-        WT_TICK(1);
         int lnext;
+        bool late = false;
         if (g.bulk) {
-            // every thread polls the copy barrier itself (bounded); a copy that never lands is flagged and
-            // the block carries on with whatever is in the buffer rather than waiting for ever
-            if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
-            WT_TICK(8);
+            // every thread polls the copy barrier itself (bounded); a copy that never lands is noticed by the
+            // whole block at the staging barrier below
+            late = !mbar_wait(bar + ring, parity, wait_limit);
             const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
             if (hoist_patch) {
                 run_patch<T, true>(sm, g, patch0, rx, nvalid);
@@ -850,8 +859,14 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         } else {
             lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, srank, nstagers);
         }
-        WT_TICK(2);
-        __syncthreads();
+        if (g.bulk) {
+            if (__syncthreads_or(late)) {
+                give_up_after_timeout(bar, g, ring, parity, u, u_end, status);
+                break;
+            }
+        } else {
+            __syncthreads();
+        }
         if (g.bulk) {
             // this ring entry is free again: refill it with the unit `nstage` ahead, behind the math
             if (tid == 0 && u + g.nstage < u_end) {
@@ -862,15 +877,13 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
         } else if (u + 1 < u_end) {  // no room for a raw buffer: at least warm the next unit in L2
-            const int cgn = fdiv(u + 1, g.d_B);
+            const int cgn = b + 1 == g.B ? cg + 1 : cg;
             if (cgn * g.NPL + g.NPL <= g.C) prefetch_unit_l2<T>(g, x, cgn * g.NPL, (u + 1) - cgn * g.B);
         }
-        WT_TICK(3);
         for (int l = lnext; l <= L; ++l) {
             stage_level(sm, g, g.offA, l);
             __syncthreads();
         }
-        WT_TICK(4);
         // ---- one item list: level tiles (Z^l = Wfold^l (*) Y^l) first, base tiles last; a thread's last
         //      item may be a base tile, which stays in registers across the barrier
         float acc[TH][4];
@@ -904,10 +917,8 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             }
         }
         const float bias = wtab[bslot * (1 + 4 * L) * WT_STRIDE + KK];
-        WT_TICK(5);
         if (g.bulk_out && tid == 0) bulk_store_wait_read();  // the previous unit's store has drained the output image
         __syncthreads();
-        WT_TICK(6);
         if (has_base) {
             const float *S = sm + bslot * g.slot_stride;
 #pragma unroll
@@ -915,13 +926,10 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             if (bslot < nvalid) store_tile<T, TH>(g, sm, out + ((size_t)b * g.C + c + bslot) * HW, bslot, tyy, txx, acc);
         }
         if (g.bulk_out) {  // the unit is contiguous in global memory: one bulk store once every tile is in place
+            fence_async_smem();  // every writer orders its shared-memory writes before the async proxy's reads
             __syncthreads();
-            if (tid == 0) {
-                fence_async_smem();
-                bulk_s2g(out + ((size_t)b * g.C + c) * HW, sm + g.out_off, (unsigned)g.NPL * g.plane_bytes);
-            }
+            if (tid == 0) bulk_s2g(out + ((size_t)b * g.C + c) * HW, sm + g.out_off, (unsigned)g.NPL * g.plane_bytes);
         }
-        WT_TICK(7);
         // The next unit's staging overwrites x / Y (last read before the barrier above) and possibly the
         // weight table (bias already in a register); Z is next written after the staging barriers.
     }
@@ -961,20 +969,24 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     for (int t = 0; t < KK; ++t) acc[t] = 0.f;
     int ring = 0;
     __syncthreads();
-    for (int u = u_begin; u < u_end; ++u) {
-        const int c = fdiv(u, g.d_B), b = u - c * g.B;  // this kernel is planned with one plane per unit: group = channel
+    int c = u_begin / g.B, b = u_begin - c * g.B;  // this kernel is planned with one plane per unit: group = channel
+    for (int u = u_begin; u < u_end; ++u, (++b == g.B ? (b = 0, ++c) : 0)) {
         int lnext;
         if (g.bulk) {
-            if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
+            const bool late = !mbar_wait(bar + ring, parity, g.no_copy ? WAIT_LIMIT_TEST : WAIT_LIMIT);
             const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
             const T *rg = reinterpret_cast<const T *>(raw + ring * g.stage_bytes + (size_t)g.NPL * g.plane_bytes);
             lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, tid, nthr);
             stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
+            if (__syncthreads_or(late)) {
+                give_up_after_timeout(bar, g, ring, parity, u, u_end, status);
+                break;
+            }
         } else {
             lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, tid, nthr);
             stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
+            __syncthreads();
         }
-        __syncthreads();
         if (g.bulk) {
             if (tid == 0 && u + g.nstage < u_end) {
                 fence_async_smem();
@@ -984,7 +996,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
         } else if (u + 1 < u_end) {
-            const int cn = fdiv(u + 1, g.d_B), bn = (u + 1) - cn * g.B;
+            const int cn = b + 1 == g.B ? c + 1 : c, bn = (u + 1) - cn * g.B;
             prefetch_unit_l2<T>(g, x, cn, bn);
             prefetch_unit_l2<T>(g, go, cn, bn);
         }
@@ -1033,7 +1045,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
             }
         }
         __syncthreads();
-        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_B) != c);
+        const bool last_of_channel = (u + 1 == u_end) || (b + 1 == g.B);
         if (last_of_channel) {
             // block tree through shared memory: every thread parks its 26 sums in the (now idle) array
             // region, then one thread per (class, tap) adds its class's threads in index order
@@ -1075,7 +1087,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 //                    closed-form synthesis of Proposition 2 and the store of grad_x.
 // Used when a unit's item list fits one round of the block (<= 256 tiles); otherwise the separate weight-
 // gradient and input-gradient kernels run.
-template <typename T, int TH, int BULK>  // BULK: tensors prefetched by bulk copy (0 none, 1 x only, 2 x and grad_out)
+template <typename T, int TH, int BULK>  // BULK: tensors prefetched by bulk copy (0 none, 2 x and grad_out)
 __global__ void __launch_bounds__(256, 2)
 plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                  const float *__restrict__ w0, const float *__restrict__ s0, const float *__restrict__ wl,
@@ -1088,7 +1100,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    if (BULK) start_prefetch<T>(bar, raw, g, x, BULK == 2 ? go : nullptr, u_begin, u_end);
+    if (BULK) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
     zero_fill(sm, g);
     unsigned parity = 0;
     const int L = g.L, nlv = g.lvl_start[L + 1], ncls = 1 + 4 * L;
@@ -1117,34 +1129,29 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     int c_prev = -1;
     int ring = 0;
     __syncthreads();
-    for (int u = u_begin; u < u_end; ++u) {
-        const int cg = fdiv(u, g.d_B), b = u - cg * g.B, c = cg * g.NPL;
+    int cg = u_begin / g.B, b = u_begin - cg * g.B;
+    for (int u = u_begin; u < u_end; ++u, (++b == g.B ? (b = 0, ++cg) : 0)) {
+        const int c = cg * g.NPL;
         const int nvalid = g.C - c < g.NPL ? g.C - c : g.NPL;
         if (c != c_prev) {
             build_weight_table(wtab, g, c, true, w0, s0, nullptr, wl, sl);
             c_prev = c;
         }
         int lnext;
+        bool late = false;
         if (BULK) {
-            if (!mbar_wait(bar + ring, parity)) atomicExch(status, 1);
+            late = !mbar_wait(bar + ring, parity, g.no_copy ? WAIT_LIMIT_TEST : WAIT_LIMIT);
             const T *rx = reinterpret_cast<const T *>(raw + ring * g.stage_bytes);
             const T *rg = reinterpret_cast<const T *>(raw + ring * g.stage_bytes + (size_t)g.NPL * g.plane_bytes);
-            const T *gg = go + ((size_t)b * g.C + c) * HW;  // grad_out straight from global memory when BULK == 1
             if (hoist_patch) {
-                // the global loads of grad_out go first so that their latency runs behind the x patches
-                if (BULK == 1) {
-                    run_patch<T, false>(sm, g, patch0, gg, nvalid, dA0, dA1, dA2);
-                    run_patch<T, false>(sm, g, patch1, gg, nvalid, dA0, dA1, dA2);
-                }
                 run_patch<T, true>(sm, g, patch0, rx, nvalid);
-                if (BULK == 2) run_patch<T, true>(sm, g, patch0, rg, nvalid, dA0, dA1, dA2);
+                run_patch<T, true>(sm, g, patch0, rg, nvalid, dA0, dA1, dA2);
                 run_patch<T, true>(sm, g, patch1, rx, nvalid);
-                if (BULK == 2) run_patch<T, true>(sm, g, patch1, rg, nvalid, dA0, dA1, dA2);
+                run_patch<T, true>(sm, g, patch1, rg, nvalid, dA0, dA1, dA2);
                 lnext = 3;
             } else {
                 lnext = stage_input<T, true>(sm, g, g.offA, rx, c, b, tid, nthr);
-                if (BULK == 2) stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
-                else stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
+                stage_input<T, true>(sm, g, g.offG, rg, c, b, tid, nthr);
             }
         } else if (hoist_patch) {
             const size_t po = ((size_t)b * g.C + c) * HW;
@@ -1155,20 +1162,27 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             lnext = stage_input<T, false>(sm, g, g.offA, x, c, b, tid, nthr);
             stage_input<T, false>(sm, g, g.offG, go, c, b, tid, nthr);
         }
-        __syncthreads();
+        if (BULK) {
+            if (__syncthreads_or(late)) {
+                give_up_after_timeout(bar, g, ring, parity, u, u_end, status);
+                break;
+            }
+        } else {
+            __syncthreads();
+        }
         if (BULK) {
             if (tid == 0 && u + g.nstage < u_end) {
                 fence_async_smem();
                 const int cgn = (u + g.nstage) / g.B;
-                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, BULK == 2 ? go : nullptr, cgn * g.NPL,
+                issue_unit_copies<T>(bar + ring, raw + ring * g.stage_bytes, g, x, go, cgn * g.NPL,
                                      (u + g.nstage) - cgn * g.B);
             }
             if (++ring == g.nstage) { ring = 0; parity ^= 1u; }
         }
-        if (BULK != 2 && u + 1 < u_end) {  // what does not come by bulk copy is warmed in L2 behind this unit's math
-            const int cgn = fdiv(u + 1, g.d_B), bn = (u + 1) - cgn * g.B;
+        if (!BULK && u + 1 < u_end) {  // no ring: the next unit is warmed in L2 behind this unit's math
+            const int cgn = b + 1 == g.B ? cg + 1 : cg, bn = (u + 1) - cgn * g.B;
             if (cgn * g.NPL + g.NPL <= g.C) {
-                if (BULK == 0) prefetch_unit_l2<T>(g, x, cgn * g.NPL, bn);
+                prefetch_unit_l2<T>(g, x, cgn * g.NPL, bn);
                 prefetch_unit_l2<T>(g, go, cgn * g.NPL, bn);
             }
         }
@@ -1240,13 +1254,11 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             if (bslot < nvalid) store_tile<T, TH>(g, sm, gx + ((size_t)b * g.C + c + bslot) * HW, bslot, tyy, txx, acc);
         }
         if (BULK && g.bulk_out) {
+            fence_async_smem();  // every writer orders its shared-memory writes before the async proxy's reads
             __syncthreads();
-            if (tid == 0) {
-                fence_async_smem();
-                bulk_s2g(gx + ((size_t)b * g.C + c) * HW, sm + g.out_off, (unsigned)g.NPL * g.plane_bytes);
-            }
+            if (tid == 0) bulk_s2g(gx + ((size_t)b * g.C + c) * HW, sm + g.out_off, (unsigned)g.NPL * g.plane_bytes);
         }
-        const bool last_of_channel = (u + 1 == u_end) || (fdiv(u + 1, g.d_B) != cg);
+        const bool last_of_channel = (u + 1 == u_end) || (b + 1 == g.B);
         if (last_of_channel) {
             // block tree through shared memory: park the 26 sums and the class of every thread in the array
             // region (idle now), then one thread per (class, tap) adds its class's threads in index order
@@ -1452,7 +1464,6 @@ inline bool plan_forward_th(int B, int C, int H, int W, int L, int elem_bytes, G
                 if (sc > best.score + 1e-9) {
                     best = cg;
                     best.smem_floats = (int)smem_floats; best.ngroups = ngroups; best.units = units;
-                    best.d_B = make_fastdiv(B);
                     best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                     found = true;
                 }
@@ -1516,7 +1527,7 @@ inline bool plan_wgrad_th(int B, int C, int H, int W, int L, int elem_bytes, Geo
                     if (sc > best.score + 1e-9) {
                         best = cg;
                         best.smem_floats = (int)smem_floats;
-                        best.ngroups = C; best.units = units; best.d_B = make_fastdiv(B);
+                        best.ngroups = C; best.units = units;
                         best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                         for (int k = 0; k <= ncls; ++k) best.thr_start[k] = thr[k];
                         int np = 1;
@@ -1559,7 +1570,7 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
         const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 20) & 1);
         bool any = false;
         // use_bulk = tensors that arrive by bulk copy: both or none (x only, with grad_out read by plain loads,
-        // is built into the kernel as BULK == 1 but measured slower than no prefetch at 56 x 56 fp32)
+        // measured slower than no prefetch at 56 x 56 fp32)
         for (int use_bulk = can_bulk ? 2 : 0; use_bulk >= 0; use_bulk -= 2) {
         Geom cg = g;
         cg.NPL = npl; cg.slot_stride = slot; cg.bulk = use_bulk;
@@ -1578,12 +1589,12 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
             if (occ > 1.0) occ = 1.0;
             const double overlap = bps >= 3 ? 1.0 : (bps == 2 ? 0.85 : 0.55);
             const double sc = teff * ((double)npl * M / (double)T) * (0.5 + 0.5 * occ) * overlap *
-                              (use_bulk == 2 ? 1.0 : (use_bulk == 1 ? 0.93 : 0.85)) *
+                              (use_bulk == 2 ? 1.0 : 0.85) *
                               partition_eff(units, nblocks) * ((double)C / ((double)ngroups * npl));
             if (sc > best.score + 1e-9) {
                 best = cg;
                 best.smem_floats = (int)smem_floats;
-                best.ngroups = ngroups; best.units = units; best.d_B = make_fastdiv(B);
+                best.ngroups = ngroups; best.units = units;
                 best.nthreads = T; best.nblocks = nblocks; best.blocks_per_sm = bps; best.score = sc;
                 int np = 1;
                 for (int ch = 0; ch < ngroups; ++ch) {
@@ -1681,6 +1692,21 @@ inline bool plan_bwd_fused(int B, int C, int H, int W, int L, int elem_bytes, Ge
 
 inline int dtype_bytes(int dtype) { return dtype == 0 ? 4 : 2; }
 
+// Human-readable launch plan of a descriptor (threads, blocks per SM, planes per unit, tile rows, ring depth).
+inline void describe(int B, int C, int H, int W, int L, int elem_bytes, unsigned tune, char *buf, size_t n) {
+    Geom f, b;
+    int o = 0;
+    if (plan_forward(B, C, H, W, L, elem_bytes, f, tune))
+        o += snprintf(buf + o, n - o, "plane fwd[T=%d bps=%d npl=%d th=%d ring=%d]", f.nthreads, f.blocks_per_sm, f.NPL, f.th,
+                      f.bulk ? f.nstage : 0);
+    if (o < (int)n && plan_bwd_fused(B, C, H, W, L, elem_bytes, b, tune))
+        snprintf(buf + o, n - o, " bwd[fused T=%d bps=%d npl=%d th=%d ring=%d np=%d]", b.nthreads, b.blocks_per_sm, b.NPL, b.th,
+                 b.bulk ? b.nstage : 0, b.np);
+    else if (o < (int)n && plan_wgrad(B, C, H, W, L, elem_bytes, b, tune))
+        snprintf(buf + o, n - o, " bwd[split wgrad T=%d bps=%d th=%d ring=%d np=%d]", b.nthreads, b.blocks_per_sm, b.th,
+                 b.bulk ? b.nstage : 0, b.np);
+}
+
 inline bool supported(int H, int W, int k, int L, int dtype) {
     if (k != 5) return false;
     Geom g;
@@ -1697,6 +1723,21 @@ inline size_t backward_workspace_bytes(int B, int C, int H, int W, int L, int el
     return STATUS_BYTES + sizeof(float) * ((size_t)C * g.np * (KK + 1) + (size_t)L * C * g.np * 4 * KK);
 }
 
+// Opt a kernel in to the large dynamic shared-memory carve-out once per device (the attribute is sticky; asking
+// for it on every launch costs host time that shows on the small layers).
+template <auto Kern>
+cudaError_t opt_in_smem() {
+    static std::atomic<unsigned long long> done{0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+    e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);
+    if (e == cudaSuccess && bit) done.fetch_or(bit, std::memory_order_release);
+    return e;
+}
+
 template <typename T, bool FLIP>
 cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *s0, const float *b0, const float *wl,
                        const float *sl, T *out, int *status, cudaStream_t st) {
@@ -1704,9 +1745,8 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
     const size_t smem = (size_t)g.smem_floats * 4;
 #define WT_LAUNCH_FWD_TH(MAXT_, MINB_, TH_)                                                         \
     {                                                                                               \
-        auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_, TH_>;                                   \
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);    \
-        if (e != cudaSuccess) return e;                                                             \
+        constexpr auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_, TH_>;                         \
+        if ((e = opt_in_smem<kern>()) != cudaSuccess) return e;                                     \
         kern<<<g.nblocks, g.nthreads, smem, st>>>(g, x, w0, s0, b0, wl, sl, out, status);           \
     }
 #define WT_LAUNCH_FWD(MAXT_, MINB_) { if (g.th == 8) WT_LAUNCH_FWD_TH(MAXT_, MINB_, 8) else WT_LAUNCH_FWD_TH(MAXT_, MINB_, 4) }
@@ -1724,9 +1764,11 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
 
 template <typename T>
 cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
-                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tune = 0) {
+                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tune = 0,
+                    bool no_copy = false) {
     Geom g;
     if (!plan_forward(B, C, H, W, L, (int)sizeof(T), g, tune)) return cudaErrorInvalidValue;
+    g.no_copy = no_copy;
     cudaError_t e = cudaMemsetAsync(ws, 0, STATUS_BYTES, st);
     if (e != cudaSuccess) return e;
     return launch_fwd<T, false>(g, x, w0, s0, b0, wl, sl, out, reinterpret_cast<int *>(ws), st);
@@ -1735,9 +1777,10 @@ cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *
 template <typename T>
 cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go, const float *w0, const float *s0,
                      const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st,
-                     unsigned tune = 0) {
+                     unsigned tune = 0, bool no_copy = false) {
     Geom gw, gf;
     if (plan_bwd_fused(B, C, H, W, L, (int)sizeof(T), gw, tune)) {
+        gw.no_copy = no_copy;
         float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
         float *partl = part0 + (size_t)C * gw.np * (KK + 1);
         const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
@@ -1745,16 +1788,15 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         if (e != cudaSuccess) return e;
 #define WT_LAUNCH_BWD(TH_, BULK_)                                                                          \
     {                                                                                                      \
-        auto kb = plane_bwd_kernel<T, TH_, BULK_>;                                                         \
-        e = cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);             \
-        if (e != cudaSuccess) return e;                                                                    \
+        constexpr auto kb = plane_bwd_kernel<T, TH_, BULK_>;                                               \
+        if ((e = opt_in_smem<kb>()) != cudaSuccess) return e;                                              \
         kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl, \
                                                                          reinterpret_cast<int *>(ws));     \
     }
         if (gw.th == 8) {
-            if (gw.bulk == 2) WT_LAUNCH_BWD(8, 2) else if (gw.bulk == 1) WT_LAUNCH_BWD(8, 1) else WT_LAUNCH_BWD(8, 0)
+            if (gw.bulk == 2) WT_LAUNCH_BWD(8, 2) else WT_LAUNCH_BWD(8, 0)
         } else {
-            if (gw.bulk == 2) WT_LAUNCH_BWD(4, 2) else if (gw.bulk == 1) WT_LAUNCH_BWD(4, 1) else WT_LAUNCH_BWD(4, 0)
+            if (gw.bulk == 2) WT_LAUNCH_BWD(4, 2) else WT_LAUNCH_BWD(4, 0)
         }
 #undef WT_LAUNCH_BWD
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -1768,6 +1810,7 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
     }
     if (!plan_wgrad(B, C, H, W, L, (int)sizeof(T), gw, tune) || !plan_forward(B, C, H, W, L, (int)sizeof(T), gf, tune))
         return cudaErrorInvalidValue;
+    gw.no_copy = gf.no_copy = no_copy;
     int *status = reinterpret_cast<int *>(ws);
     float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
     float *partl = part0 + (size_t)C * gw.np * (KK + 1);
@@ -1777,9 +1820,8 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
     const size_t smem = (size_t)gw.smem_floats * 4;
 #define WT_LAUNCH_WG(MAXT_, MINB_, TH_)                                                            \
     {                                                                                              \
-        auto kw = plane_wgrad_kernel<T, MAXT_, MINB_, TH_>;                                        \
-        e = cudaFuncSetAttribute(kw, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT);     \
-        if (e != cudaSuccess) return e;                                                            \
+        constexpr auto kw = plane_wgrad_kernel<T, MAXT_, MINB_, TH_>;                              \
+        if ((e = opt_in_smem<kw>()) != cudaSuccess) return e;                                      \
         kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);                \
     }
     if (gw.nthreads <= 128) {

@@ -214,7 +214,7 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
     if (use_plane_path(d)) {
         if constexpr (K == 5)
             return wt::plane::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws,
-                                         st, d->flags >> 8) == cudaSuccess
+                                         st, d->flags >> 8, (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
@@ -229,7 +229,8 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
         if constexpr (K == 5) {
             wt::EpiloguePtrs ep = {};
             if (wt::plane::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl,
-                                       (T *)gx, ws, &ep, st, d->flags >> 8) != cudaSuccess)
+                                       (T *)gx, ws, &ep, st, d->flags >> 8,
+                                       (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
         }
@@ -329,6 +330,23 @@ wtconv_status side_stream_for_current_device(cudaStream_t *out, int which = 0) {
     return WTCONV_OK;
 }
 
+// Events of wtconv_step_host, per device, created on first use and kept for the process (calls on one device
+// must not overlap in time, so they can share them; creating and destroying twenty events per call costs more
+// host time than a small layer's kernels take).
+constexpr int STEP_EVENTS = 2 * STEP_MAX_CHUNKS + 4;
+cudaEvent_t g_step_events[MAX_DEVICES][STEP_EVENTS] = {};
+wtconv_status step_events_for_current_device(cudaEvent_t **out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return WTCONV_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    for (int i = 0; i < STEP_EVENTS; ++i)
+        if (!g_step_events[dev][i] &&
+            cudaEventCreateWithFlags(&g_step_events[dev][i], cudaEventDisableTiming) != cudaSuccess)
+            return WTCONV_ERR_CUDA;
+    *out = g_step_events[dev];
+    return WTCONV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -372,6 +390,18 @@ wtconv_status wtconv_workspace_bytes(const wtconv_desc *d, size_t *fwd_bytes, si
 const char *wtconv_plan_name(const wtconv_desc *d) {
     if (validate_desc(d) != WTCONV_OK) return nullptr;
     return use_plane_path(d) ? "plane" : "tiled";
+}
+
+wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
+    wtconv_status st = validate_desc(d);
+    if (st != WTCONV_OK) return st;
+    if (!buf || n == 0) return WTCONV_ERR_NULL;
+    buf[0] = 0;
+    if (use_plane_path(d))
+        wt::plane::describe(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), d->flags >> 8, buf, n);
+    else
+        snprintf(buf, n, "tiled fwd[%d launches] bwd[%d launches]", d->L + 1, d->L + 2);
+    return WTCONV_OK;
 }
 
 wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *bwd) {
@@ -441,8 +471,18 @@ wtconv_status wtconv_step_host_workspace_bytes(const wtconv_desc *d, size_t *byt
     ParamSizes ps = param_sizes(d);
     const size_t par = align_up(ps.w0) + 2 * align_up(ps.s0) + align_up(ps.wl) + align_up(ps.sl);
     size_t f = fwd_ws_bytes(d), b = bwd_ws_bytes(d);
+    size_t scratch = f > b ? f : b;
+    const int nch = pick_step_chunks(d);
+    if (nch > 1) {  // the pipelined step runs the kernels on B / nch images: their scratch need not be smaller
+        wtconv_desc dc = *d;
+        dc.B = d->B / nch;
+        f = fwd_ws_bytes(&dc);
+        b = bwd_ws_bytes(&dc);
+        if (f > scratch) scratch = f;
+        if (b > scratch) scratch = b;
+    }
     // parameters, their gradients, and one more gradient set per batch chunk of the pipelined step
-    *bytes = 4 * act + (2 + STEP_MAX_CHUNKS) * par + (f > b ? f : b);
+    *bytes = 4 * act + (2 + STEP_MAX_CHUNKS) * par + align_up(scratch);
     return WTCONV_OK;
 }
 
@@ -482,17 +522,9 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     // way up (the link is full duplex), and `stream` waits for that copy before it reaches the end of the step.
     cudaStream_t side = nullptr;
     if ((st = side_stream_for_current_device(&side)) != WTCONV_OK) return st;
-    cudaEvent_t fwd_done = nullptr, out_home = nullptr;
-    if (cudaEventCreateWithFlags(&fwd_done, cudaEventDisableTiming) != cudaSuccess) return WTCONV_ERR_CUDA;
-    if (cudaEventCreateWithFlags(&out_home, cudaEventDisableTiming) != cudaSuccess) {
-        cudaEventDestroy(fwd_done);
-        return WTCONV_ERR_CUDA;
-    }
-    // the events are released as soon as the work recorded so far has passed them
-    struct EventGuard {
-        cudaEvent_t a, b;
-        ~EventGuard() { cudaEventDestroy(a); cudaEventDestroy(b); }
-    } guard = {fwd_done, out_home};
+    cudaEvent_t *pool = nullptr;
+    if ((st = step_events_for_current_device(&pool)) != WTCONV_OK) return st;
+    cudaEvent_t fwd_done = pool[STEP_EVENTS - 2], out_home = pool[STEP_EVENTS - 1];
     const float *b0p = h_b0 ? b0 : nullptr;
     const int nch = pick_step_chunks(d);
     if (nch > 1) {
@@ -513,13 +545,7 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
         h2d(sl, h_sl, ps.sl);
         // events: [0..nch) chunk computed, [nch] downloads done, [nch+1] stream position at entry,
         // [nch+2 .. 2 nch+2) chunk uploaded
-        constexpr int NEV = 2 * STEP_MAX_CHUNKS + 2;
-        cudaEvent_t ev[NEV] = {};
-        struct EventsGuard {
-            cudaEvent_t *e;
-            ~EventsGuard() { for (int i = 0; i < NEV; ++i) if (e[i]) cudaEventDestroy(e[i]); }
-        } eguard = {ev};
-        for (int c = 0; c < 2 * nch + 2 && ok; ++c) ok = cudaEventCreateWithFlags(&ev[c], cudaEventDisableTiming) == cudaSuccess;
+        cudaEvent_t *ev = pool;
         cudaStream_t up = nullptr;
         if (ok && side_stream_for_current_device(&up, 1) != WTCONV_OK) ok = false;
         if (!ok) return WTCONV_ERR_CUDA;
@@ -604,7 +630,13 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
 wtconv_status wtconv_read_status(const wtconv_desc *d, const void *workspace, int32_t *h_flag, void *stream) {
     wtconv_status st = validate_desc(d);
     if (st != WTCONV_OK) return st;
-    if (!workspace || !h_flag) return WTCONV_ERR_NULL;
+    if (!h_flag) return WTCONV_ERR_NULL;
+    if (!workspace) {  // the scratch array built into the library (wtconv_backward_static)
+        void *scratch = nullptr;
+        if ((st = check_device()) != WTCONV_OK) return st;
+        if ((st = static_scratch_for_current_device(&scratch)) != WTCONV_OK) return st;
+        workspace = scratch;
+    }
     if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
     if (!use_plane_path(d)) {  // the tiled kernels wait for nothing and keep no status word
         *h_flag = 0;
@@ -623,6 +655,7 @@ wtconv_status wtconv_backward_static(const wtconv_desc *d, const void *x, const 
     wtconv_status st = validate_desc(d);
     if (st != WTCONV_OK) return st;
     if (bwd_ws_bytes(d) > (size_t)WTCONV_STATIC_SCRATCH_BYTES) return WTCONV_ERR_WORKSPACE;  // shape needs more scratch than is built in
+    if ((st = check_device()) != WTCONV_OK) return st;
     void *scratch = nullptr;
     if ((st = static_scratch_for_current_device(&scratch)) != WTCONV_OK) return st;
     // wtconv_backward clears the parts of its workspace that must start at zero on every call, so the
@@ -630,15 +663,5 @@ wtconv_status wtconv_backward_static(const wtconv_desc *d, const void *x, const 
     return wtconv_backward(d, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad_s0, grad_b0, grad_wl, grad_sl,
                            scratch, (size_t)WTCONV_STATIC_SCRATCH_BYTES, stream);
 }
-
-#ifdef WT_PHASE_TIMING
-// working probe only (never part of the shipped library): read and clear the per-phase cycle counters
-int wtconv_debug_phase_cycles(unsigned long long *out16) {
-    cudaDeviceSynchronize();
-    unsigned long long z[32] = {0};
-    if (cudaMemcpyFromSymbol(out16, wt::plane::wt_phase_cycles, sizeof(z)) != cudaSuccess) return 1;
-    return cudaMemcpyToSymbol(wt::plane::wt_phase_cycles, z, sizeof(z)) != cudaSuccess;
-}
-#endif
 
 }  // extern "C"

@@ -15,10 +15,12 @@ LIB_PATH = os.path.join(_HERE, "libwtconv_b200.so")
 
 F32, F16, BF16 = 0, 1, 2
 FLAG_TILED_ONLY = 1
+FLAG_TEST_NO_COPY = 2
+ARITHMETIC_DTYPE = "f32"  # every kernel multiplies and accumulates in float32, whatever the storage type
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_NAMES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
 
-EXPORTS = ["wtconv_status_string", "wtconv_level_shape", "wtconv_workspace_bytes", "wtconv_plan_name",
+EXPORTS = ["wtconv_status_string", "wtconv_level_shape", "wtconv_workspace_bytes", "wtconv_plan_name", "wtconv_plan_describe",
            "wtconv_launch_count", "wtconv_forward", "wtconv_backward", "wtconv_read_status", "wtconv_backward_static",
            "wtconv_step_host_workspace_bytes", "wtconv_step_host"]
 
@@ -50,6 +52,7 @@ def lib():
         L.wtconv_status_string.argtypes = [ctypes.c_int]
         L.wtconv_plan_name.restype = ctypes.c_char_p
         L.wtconv_plan_name.argtypes = [dp]
+        L.wtconv_plan_describe.argtypes = [dp, ctypes.c_char_p, sz]
         L.wtconv_level_shape.argtypes = [dp, ctypes.c_int, i32p, i32p]
         L.wtconv_workspace_bytes.argtypes = [dp, ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.wtconv_launch_count.argtypes = [dp, i32p, i32p]
@@ -91,6 +94,12 @@ def wtconv_plan_name(desc):
     return None if r is None else r.decode()
 
 
+def wtconv_plan_describe(desc):
+    buf = ctypes.create_string_buffer(256)
+    _check(lib().wtconv_plan_describe(ctypes.byref(desc), buf, 256))
+    return buf.value.decode()
+
+
 def wtconv_launch_count(desc):
     f, b = ctypes.c_int32(), ctypes.c_int32()
     _check(lib().wtconv_launch_count(ctypes.byref(desc), ctypes.byref(f), ctypes.byref(b)))
@@ -130,7 +139,8 @@ def wtconv_backward(desc, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad
 
 
 def wtconv_read_status(desc, workspace, h_flag, stream=None):
-    """Enqueue a copy of the workspace's device status word into the host int32 tensor `h_flag` (pin it)."""
+    """Enqueue a copy of the workspace's device status word into the host int32 tensor `h_flag` (pin it).
+    `workspace=None` reads the array built into the library (the one wtconv_backward_static uses)."""
     _need_cuda(workspace)
     if h_flag.is_cuda or h_flag.dtype != torch.int32 or h_flag.numel() < 1:
         raise ValueError("h_flag must be a host int32 tensor")
@@ -187,6 +197,12 @@ def forward_backward(desc, x, g, w0, s0, b0, wl, sl, workspace=None, stream=None
         gwl, gsl = torch.empty_like(wl), torch.empty_like(sl)
     else:
         gwl = gsl = None
+    flags = torch.zeros(2, dtype=torch.int32).pin_memory()
     wtconv_forward(desc, x, w0, s0, b0, wl, sl, out, ws, stream)
+    wtconv_read_status(desc, ws, flags[0:1], stream)
     wtconv_backward(desc, x, g, w0, s0, b0, wl, sl, gx, gw0, gs0, gb0, gwl, gsl, ws, stream)
+    wtconv_read_status(desc, ws, flags[1:2], stream)
+    (torch.cuda.current_stream() if stream is None else stream).synchronize()
+    if int(flags[0]) or int(flags[1]):  # a bounded device-side wait ran out: the outputs are not valid
+        raise WTConvError(11, lib().wtconv_status_string(11).decode())
     return out, dict(dx=gx, dw0=gw0, ds0=gs0, db0=gb0, dwl=gwl, dsl=gsl)
