@@ -76,6 +76,18 @@ typedef enum {
  * limit is tiny, so every wait for a copy runs out; the kernels record it in the status word and return
  * normally with nothing in flight (outputs are then invalid by design).  Never set it in production. */
 #define WTCONV_FLAG_TEST_NO_COPY 2u
+#define WTCONV_FLAG_NO_TEAM 4u /* never take the team kernels for small planes (used to test the block-per-plane kernels on them) */
+/* Comparator: run the layer as the chain of separate operators of Sec. 3.1 (analysis, depthwise conv, scale pass,
+ * slice, add, concatenate, synthesis per level; base conv, scale pass, add), every intermediate in HBM, as plain
+ * kernels of this library.  It is what the paper measures its fused kernels against (Eq. 2 vs Eq. 10, Tables 1-3);
+ * in this mode wtconv_backward first re-runs the forward chain (the autograd tape) and then every operator's
+ * gradient as its own launch, so it costs one reference training step.  Two further bits reproduce the cumulative
+ * ablation of Table 8 on the forward chain: FUSED_ANALYSIS (butterfly on chip in the level conv kernel, Sec. 4.1),
+ * COLLAPSED_SYNTHESIS (one closed-form pass, Sec. 4.2); with scale folding (Sec. 4.3) added on top the chain is
+ * the paper's fused design = WTCONV_FLAG_TILED_ONLY.  Workspace sizes are far larger in this mode (query them). */
+#define WTCONV_FLAG_REFERENCE_CHAIN 8u
+#define WTCONV_FLAG_ABLATE_FUSED_ANALYSIS 16u
+#define WTCONV_FLAG_ABLATE_COLLAPSED_SYNTHESIS 32u
 /* Launch-plan overrides for the plane-resident kernels, for tuning experiments (0 = let the planner choose):
  *   bits  8-12  threads per block / 32 of the forward / input-gradient kernel
  *   bits 13-15  resident blocks per SM of that kernel
@@ -111,8 +123,9 @@ wtconv_status wtconv_level_shape(const wtconv_desc *desc, int level, int32_t *Hl
  * Either output pointer may be NULL. */
 wtconv_status wtconv_workspace_bytes(const wtconv_desc *desc, size_t *fwd_bytes, size_t *bwd_bytes);
 
-/* Name of the kernel family a descriptor dispatches to ("plane" = whole-plane shared-memory
- * kernels, "tiled" = per-level tiled kernels).  Host call; returns NULL for an invalid desc. */
+/* Name of the kernel family a descriptor dispatches to ("team" = small planes, several per thread team; "plane" =
+ * one block per whole plane in shared memory; "tiled" = per-level tiled kernels).  Host call; returns NULL for
+ * an invalid desc. */
 const char *wtconv_plan_name(const wtconv_desc *desc);
 
 /* Launch plan of a descriptor as text (threads per block, resident blocks per SM, planes per work unit, register

@@ -1841,5 +1841,14 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
     return cudaSuccess;
 }
 
+// Explicit instantiation (EXTERN empty) or its declaration (EXTERN = extern) of the host entry points for one
+// activation type: the kernels are compiled once, in the instantiation unit of that type.
+#define WT_PLANE_INSTANTIATE(T, EXTERN)                                                                                    \
+    EXTERN template cudaError_t forward<T>(int, int, int, int, int, const T *, const float *, const float *, const float *, \
+                                           const float *, const float *, T *, char *, cudaStream_t, unsigned, bool);       \
+    EXTERN template cudaError_t backward<T>(int, int, int, int, int, const T *, const T *, const float *, const float *,    \
+                                            const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t,       \
+                                            unsigned, bool);
+
 }  // namespace plane
 }  // namespace wt

@@ -814,6 +814,7 @@ struct EpiloguePtrs {
     int npl[8];
 };
 
+template <int UNUSED>  // a template only so that every translation unit may include this header
 __global__ void __launch_bounds__(128)
 unfold_epilogue_kernel(int C, int K, int L, EpiloguePtrs ep, const float *__restrict__ w0,
                        const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,

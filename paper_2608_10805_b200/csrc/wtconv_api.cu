@@ -1,24 +1,55 @@
 // C ABI of the WTConv library: validation, workspace planning and kernel dispatch.
-// Declarations and the full contract are in include/wtconv.h.
+// Declarations and the full contract are in include/wtconv.h.  The kernels themselves are compiled in the
+// per-dtype instantiation units (inst_*.cu); this unit only declares those instantiations.
 #include "../../include/wtconv.h"
 
 #include "common.cuh"
 #include "tiled_kernels.cuh"
 #include "plane_kernels.cuh"
+#include "team_kernels.cuh"
+#include "tiled_host.cuh"
+#include "reference_chain.cuh"
 
 #include <mutex>
 
+namespace wt {
+namespace plane {
+WT_PLANE_INSTANTIATE(float, extern)
+WT_PLANE_INSTANTIATE(__half, extern)
+WT_PLANE_INSTANTIATE(__nv_bfloat16, extern)
+}  // namespace plane
+namespace team {
+WT_TEAM_INSTANTIATE(float, extern)
+WT_TEAM_INSTANTIATE(__half, extern)
+WT_TEAM_INSTANTIATE(__nv_bfloat16, extern)
+}  // namespace team
+namespace host {
+WT_TILED_INSTANTIATE(float, 3, extern)
+WT_TILED_INSTANTIATE(float, 5, extern)
+WT_TILED_INSTANTIATE(float, 7, extern)
+WT_TILED_INSTANTIATE(__half, 3, extern)
+WT_TILED_INSTANTIATE(__half, 5, extern)
+WT_TILED_INSTANTIATE(__half, 7, extern)
+WT_TILED_INSTANTIATE(__nv_bfloat16, 3, extern)
+WT_TILED_INSTANTIATE(__nv_bfloat16, 5, extern)
+WT_TILED_INSTANTIATE(__nv_bfloat16, 7, extern)
+}  // namespace host
+namespace refchain {
+WT_REFCHAIN_INSTANTIATE(float, 3, extern)
+WT_REFCHAIN_INSTANTIATE(float, 5, extern)
+WT_REFCHAIN_INSTANTIATE(float, 7, extern)
+WT_REFCHAIN_INSTANTIATE(__half, 3, extern)
+WT_REFCHAIN_INSTANTIATE(__half, 5, extern)
+WT_REFCHAIN_INSTANTIATE(__half, 7, extern)
+WT_REFCHAIN_INSTANTIATE(__nv_bfloat16, 3, extern)
+WT_REFCHAIN_INSTANTIATE(__nv_bfloat16, 5, extern)
+WT_REFCHAIN_INSTANTIATE(__nv_bfloat16, 7, extern)
+}  // namespace refchain
+}  // namespace wt
+
 namespace {
 
-using wt::host_half_up;
-
-constexpr size_t ALIGN = 256;
-inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
-inline int cdiv(int a, int b) { return (a + b - 1) / b; }
-
-struct Shapes {
-    int Hs[WTCONV_MAX_LEVELS + 1], Ws[WTCONV_MAX_LEVELS + 1];
-};
+using namespace wt::host;
 
 wtconv_status validate_desc(const wtconv_desc *d) {
     if (!d) return WTCONV_ERR_NULL;
@@ -28,79 +59,6 @@ wtconv_status validate_desc(const wtconv_desc *d) {
     if (d->L < 0 || d->L > WTCONV_MAX_LEVELS) return WTCONV_ERR_LEVELS;
     if (d->dtype != WTCONV_F32 && d->dtype != WTCONV_F16 && d->dtype != WTCONV_BF16) return WTCONV_ERR_DTYPE;
     return WTCONV_OK;
-}
-
-Shapes level_shapes(const wtconv_desc *d) {
-    Shapes s;
-    s.Hs[0] = d->H;
-    s.Ws[0] = d->W;
-    for (int l = 1; l <= WTCONV_MAX_LEVELS; ++l) {
-        s.Hs[l] = host_half_up(s.Hs[l - 1]);
-        s.Ws[l] = host_half_up(s.Ws[l - 1]);
-    }
-    return s;
-}
-
-size_t elem_bytes(int dtype) { return dtype == WTCONV_F32 ? 4 : 2; }
-
-// ------------------------------------------------------------------ tiled-path workspace plan
-struct TiledPlan {
-    Shapes sh;
-    int P, KK;
-    // forward
-    size_t z_off[WTCONV_MAX_LEVELS], xc_off[WTCONV_MAX_LEVELS];  // Z^l / dY^l and carrier X^l (index l-1)
-    size_t fwd_bytes;
-    // backward extras
-    size_t gc_off[WTCONV_MAX_LEVELS];
-    size_t part0_off, partl_off[WTCONV_MAX_LEVELS];
-    int bsplit0, np0, bsplitl[WTCONV_MAX_LEVELS], npl[WTCONV_MAX_LEVELS];
-    int tx0, ty0, txl[WTCONV_MAX_LEVELS], tyl[WTCONV_MAX_LEVELS];
-    size_t bwd_bytes;
-};
-
-int pick_bsplit(int B, long long blocks_per_batchloop) {
-    // enough blocks to fill 148 SMs several times over, but never more than one batch per block
-    long long want = (4LL * 148 * 2 + blocks_per_batchloop - 1) / blocks_per_batchloop;
-    if (want < 1) want = 1;
-    if (want > B) want = B;
-    return (int)want;
-}
-
-TiledPlan make_tiled_plan(const wtconv_desc *d) {
-    TiledPlan p;
-    p.sh = level_shapes(d);
-    p.P = d->B * d->C;
-    p.KK = d->k * d->k;
-    size_t off = 0;
-    for (int l = 1; l <= d->L; ++l) {
-        size_t S = (size_t)p.sh.Hs[l] * p.sh.Ws[l];
-        p.z_off[l - 1] = off;
-        off = align_up(off + sizeof(float) * 4 * S * p.P);
-        p.xc_off[l - 1] = off;
-        if (l < d->L) off = align_up(off + sizeof(float) * S * p.P);
-    }
-    p.fwd_bytes = off;
-    for (int l = 1; l < d->L; ++l) {
-        size_t S = (size_t)p.sh.Hs[l] * p.sh.Ws[l];
-        p.gc_off[l - 1] = off;
-        off = align_up(off + sizeof(float) * S * p.P);
-    }
-    p.tx0 = cdiv(d->W, wt::tiled::STW);
-    p.ty0 = cdiv(d->H, wt::tiled::STH);
-    p.bsplit0 = pick_bsplit(d->B, (long long)p.tx0 * p.ty0 * d->C);
-    p.np0 = p.tx0 * p.ty0 * p.bsplit0;
-    p.part0_off = off;
-    off = align_up(off + sizeof(float) * (size_t)d->C * p.np0 * (p.KK + 1));
-    for (int l = 1; l <= d->L; ++l) {
-        p.txl[l - 1] = cdiv(p.sh.Ws[l], wt::tiled::TW);
-        p.tyl[l - 1] = cdiv(p.sh.Hs[l], wt::tiled::TH);
-        p.bsplitl[l - 1] = pick_bsplit(d->B, (long long)p.txl[l - 1] * p.tyl[l - 1] * d->C);
-        p.npl[l - 1] = p.txl[l - 1] * p.tyl[l - 1] * p.bsplitl[l - 1];
-        p.partl_off[l - 1] = off;
-        off = align_up(off + sizeof(float) * (size_t)d->C * p.npl[l - 1] * 4 * p.KK);
-    }
-    p.bwd_bytes = off;
-    return p;
 }
 
 bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
@@ -116,101 +74,30 @@ wtconv_status check_device() {
     return major == 10 ? WTCONV_OK : WTCONV_ERR_ARCH;
 }
 
-inline wtconv_status launch_status() { return cudaGetLastError() == cudaSuccess ? WTCONV_OK : WTCONV_ERR_CUDA; }
-
-// ------------------------------------------------------------------ tiled forward / backward
-template <typename T, int K>
-wtconv_status tiled_forward(const wtconv_desc *d, const T *x, const float *w0, const float *s0, const float *b0,
-                            const float *wl, const float *sl, T *out, char *ws, cudaStream_t st) {
-    using namespace wt::tiled;
-    TiledPlan pl = make_tiled_plan(d);
-    wt::tiled::LevelPtrs lv = {};
-    const int C = d->C, KK = K * K;
-    for (int l = 1; l <= d->L; ++l) {
-        const int Hp = pl.sh.Hs[l - 1], Wp = pl.sh.Ws[l - 1], Hl = pl.sh.Hs[l], Wl = pl.sh.Ws[l];
-        float *Z = (float *)(ws + pl.z_off[l - 1]);
-        float *Xl = (l < d->L) ? (float *)(ws + pl.xc_off[l - 1]) : nullptr;
-        dim3 grid((unsigned)((size_t)pl.P * cdiv(Wl, TW) * cdiv(Hl, TH)));  // plane-major
-        const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
-        if (l == 1)
-            level_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, Hp, Wp, Hl, Wl, C, wq, sq, Z, Xl);
-        else
-            level_fwd_kernel<float, K><<<grid, NTHREADS, 0, st>>>((const float *)(ws + pl.xc_off[l - 2]), Hp, Wp, Hl,
-                                                                   Wl, C, wq, sq, Z, Xl);
-        lv.z[l - 1] = Z;
-        lv.Hl[l - 1] = Hl;
-        lv.Wl[l - 1] = Wl;
-    }
-    dim3 grid((unsigned)((size_t)pl.P * cdiv(d->W, STW) * cdiv(d->H, STH)));  // plane-major
-    synth_fwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, d->H, d->W, C, d->L, w0, s0, b0, lv, out);
-    return launch_status();
-}
-
-wtconv_status launch_epilogue(const wtconv_desc *d, const wt::EpiloguePtrs &ep, const float *w0, const float *s0,
-                              const float *b0, const float *wl, const float *sl, float *gw0, float *gs0, float *gb0,
-                              float *gwl, float *gsl, cudaStream_t st) {
-    const int KK = d->k * d->k;
-    size_t smem = sizeof(double) * (KK + 1 + (size_t)d->L * 4 * KK);
-    wt::unfold_epilogue_kernel<<<d->C, 128, smem, st>>>(d->C, d->k, d->L, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl,
-                                                        gsl);
-    return launch_status();
-}
-
-template <typename T, int K>
-wtconv_status tiled_backward(const wtconv_desc *d, const T *x, const T *g, const float *w0, const float *s0,
-                             const float *b0, const float *wl, const float *sl, T *gx, float *gw0, float *gs0,
-                             float *gb0, float *gwl, float *gsl, char *ws, cudaStream_t st) {
-    using namespace wt::tiled;
-    TiledPlan pl = make_tiled_plan(d);
-    wt::tiled::LevelPtrs lv = {};
-    wt::EpiloguePtrs ep = {};
-    const int C = d->C, KK = K * K;
-    for (int l = 1; l <= d->L; ++l) {
-        const int Hp = pl.sh.Hs[l - 1], Wp = pl.sh.Ws[l - 1], Hl = pl.sh.Hs[l], Wl = pl.sh.Ws[l];
-        float *dY = (float *)(ws + pl.z_off[l - 1]);
-        float *Xl = (l < d->L) ? (float *)(ws + pl.xc_off[l - 1]) : nullptr;
-        float *Gl = (l < d->L) ? (float *)(ws + pl.gc_off[l - 1]) : nullptr;
-        float *part = (float *)(ws + pl.partl_off[l - 1]);
-        dim3 grid((unsigned)((size_t)C * pl.bsplitl[l - 1] * pl.txl[l - 1] * pl.tyl[l - 1]));  // (channel, part)-major
-        const float *wq = wl + (size_t)(l - 1) * C * 4 * KK, *sq = sl + (size_t)(l - 1) * C * 4;
-        constexpr size_t lsmem = level_bwd_smem_bytes<K>();  // above 48 KB for k = 7: opt in
-        if (l == 1) {
-            auto kern = level_bwd_kernel<T, K>;
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsmem) != cudaSuccess)
-                return WTCONV_ERR_CUDA;
-            kern<<<grid, NTHREADS, lsmem, st>>>(x, g, Hp, Wp, Hl, Wl, d->B, C, pl.bsplitl[l - 1], wq, sq, dY, Xl, Gl, part);
-        } else {
-            auto kern = level_bwd_kernel<float, K>;
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lsmem) != cudaSuccess)
-                return WTCONV_ERR_CUDA;
-            kern<<<grid, NTHREADS, lsmem, st>>>((const float *)(ws + pl.xc_off[l - 2]), (const float *)(ws + pl.gc_off[l - 2]),
-                                                Hp, Wp, Hl, Wl, d->B, C, pl.bsplitl[l - 1], wq, sq, dY, Xl, Gl, part);
-        }
-        lv.z[l - 1] = dY;
-        lv.Hl[l - 1] = Hl;
-        lv.Wl[l - 1] = Wl;
-        ep.partl[l - 1] = part;
-        ep.npl[l - 1] = pl.npl[l - 1];
-    }
-    float *part0 = (float *)(ws + pl.part0_off);
-    dim3 grid((unsigned)((size_t)C * pl.bsplit0 * pl.tx0 * pl.ty0));  // (channel, part)-major
-    synth_bwd_kernel<T, K><<<grid, NTHREADS, 0, st>>>(x, g, d->H, d->W, d->B, C, d->L, pl.bsplit0, w0, s0, lv, gx,
-                                                      part0);
-    ep.part0 = part0;
-    ep.np0 = pl.np0;
-    if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
-    return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
-}
-
 // ------------------------------------------------------------------ dispatch
-bool use_plane_path(const wtconv_desc *d) {
-    if (d->flags & WTCONV_FLAG_TILED_ONLY) return false;
-    return wt::plane::supported(d->H, d->W, d->k, d->L, d->dtype);
+int team_force_g(const wtconv_desc *d) { return (int)((d->flags >> 16) & 63u); }  // "planes per work unit" override
+bool use_ref_chain(const wtconv_desc *d) { return (d->flags & WTCONV_FLAG_REFERENCE_CHAIN) != 0; }
+bool use_team_path(const wtconv_desc *d) {
+    if (d->flags & (WTCONV_FLAG_TILED_ONLY | WTCONV_FLAG_NO_TEAM | WTCONV_FLAG_REFERENCE_CHAIN)) return false;
+    if ((d->flags >> 8) & ~(63u << 8)) return false;  // other launch-plan overrides address the block-per-plane kernels
+    return wt::team::supported(d->B, d->C, d->H, d->W, d->k, d->L, d->dtype, team_force_g(d));
+}
+bool use_plane_path(const wtconv_desc *d) {  // any kernel family that keeps whole planes on chip (and a status word)
+    if (d->flags & (WTCONV_FLAG_TILED_ONLY | WTCONV_FLAG_REFERENCE_CHAIN)) return false;
+    return use_team_path(d) || wt::plane::supported(d->H, d->W, d->k, d->L, d->dtype);
 }
 
 template <typename T, int K>
 wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, const float *s0, const float *b0,
                          const float *wl, const float *sl, void *out, char *ws, cudaStream_t st) {
+    if (use_ref_chain(d)) return wt::refchain::forward<T, K>(d, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st);
+    if constexpr (K == 5) {
+        if (use_team_path(d))
+            return wt::team::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st,
+                                        (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, team_force_g(d)) == cudaSuccess
+                       ? WTCONV_OK
+                       : WTCONV_ERR_CUDA;
+    }
     if (use_plane_path(d)) {
         if constexpr (K == 5)
             return wt::plane::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws,
@@ -225,6 +112,18 @@ template <typename T, int K>
 wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, const float *w0, const float *s0,
                           const float *b0, const float *wl, const float *sl, void *gx, float *gw0, float *gs0,
                           float *gb0, float *gwl, float *gsl, char *ws, cudaStream_t st) {
+    if (use_ref_chain(d))
+        return wt::refchain::backward<T, K>(d, (const T *)x, (const T *)g, w0, s0, b0, wl, sl, (T *)gx, gw0, gs0, gb0, gwl, gsl,
+                                            ws, st);
+    if constexpr (K == 5) {
+        if (use_team_path(d)) {
+            wt::EpiloguePtrs ep = {};
+            if (wt::team::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl, (T *)gx,
+                                      ws, &ep, st, (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, team_force_g(d)) != cudaSuccess)
+                return WTCONV_ERR_CUDA;
+            return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
+        }
+    }
     if (use_plane_path(d)) {
         if constexpr (K == 5) {
             wt::EpiloguePtrs ep = {};
@@ -256,10 +155,13 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
     } while (0)
 
 size_t fwd_ws_bytes(const wtconv_desc *d) {
+    if (use_ref_chain(d)) return wt::refchain::make_plan(d).fwd_bytes;
     if (use_plane_path(d)) return align_up(wt::plane::forward_workspace_bytes(d->B, d->C, d->H, d->W, d->L));
     return make_tiled_plan(d).fwd_bytes;
 }
 size_t bwd_ws_bytes(const wtconv_desc *d) {
+    if (use_ref_chain(d)) return wt::refchain::make_plan(d).bwd_bytes;
+    if (use_team_path(d)) return align_up(wt::team::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), team_force_g(d)));
     if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), d->flags >> 8));
     return make_tiled_plan(d).bwd_bytes;
 }
@@ -389,7 +291,7 @@ wtconv_status wtconv_workspace_bytes(const wtconv_desc *d, size_t *fwd_bytes, si
 
 const char *wtconv_plan_name(const wtconv_desc *d) {
     if (validate_desc(d) != WTCONV_OK) return nullptr;
-    return use_plane_path(d) ? "plane" : "tiled";
+    return use_ref_chain(d) ? "reference-chain" : use_team_path(d) ? "team" : use_plane_path(d) ? "plane" : "tiled";
 }
 
 wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
@@ -397,7 +299,13 @@ wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
     if (st != WTCONV_OK) return st;
     if (!buf || n == 0) return WTCONV_ERR_NULL;
     buf[0] = 0;
-    if (use_plane_path(d))
+    if (use_ref_chain(d))
+        snprintf(buf, n, "reference-chain (separate operators, intermediates in HBM)%s%s",
+                 (d->flags & WTCONV_FLAG_ABLATE_FUSED_ANALYSIS) ? " +fused-analysis" : "",
+                 (d->flags & WTCONV_FLAG_ABLATE_COLLAPSED_SYNTHESIS) ? " +collapsed-synthesis" : "");
+    else if (use_team_path(d))
+        wt::team::describe(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), buf, n, team_force_g(d));
+    else if (use_plane_path(d))
         wt::plane::describe(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), d->flags >> 8, buf, n);
     else
         snprintf(buf, n, "tiled fwd[%d launches] bwd[%d launches]", d->L + 1, d->L + 2);
@@ -407,7 +315,15 @@ wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
 wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *bwd) {
     wtconv_status st = validate_desc(d);
     if (st != WTCONV_OK) return st;
-    if (use_plane_path(d)) {
+    if (use_ref_chain(d)) {
+        const bool fa = d->flags & WTCONV_FLAG_ABLATE_FUSED_ANALYSIS, cs = d->flags & WTCONV_FLAG_ABLATE_COLLAPSED_SYNTHESIS;
+        const int nf = (fa ? 1 : 0) + d->L * (fa ? 2 : 3) + (d->L > 1 && !fa ? d->L - 1 : 0) + 2 + (cs ? 1 : 2 * d->L + 1);
+        if (fwd) *fwd = nf;
+        if (bwd) *bwd = (4 * d->L + 3) + 7 + 9 * d->L;  // plain forward chain + gradient launches (approximate for L > 1 slices)
+    } else if (use_team_path(d)) {
+        if (fwd) *fwd = 1;
+        if (bwd) *bwd = 2;  // fused backward + epilogue (plus one memset node)
+    } else if (use_plane_path(d)) {
         if (fwd) *fwd = 1;
         if (bwd) {
             wt::plane::Geom gq;

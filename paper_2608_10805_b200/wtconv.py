@@ -16,6 +16,10 @@ LIB_PATH = os.path.join(_HERE, "libwtconv_b200.so")
 F32, F16, BF16 = 0, 1, 2
 FLAG_TILED_ONLY = 1
 FLAG_TEST_NO_COPY = 2
+FLAG_NO_TEAM = 4
+FLAG_REFERENCE_CHAIN = 8            # comparator: the layer as separate operators with every intermediate in HBM
+FLAG_ABLATE_FUSED_ANALYSIS = 16     # (with FLAG_REFERENCE_CHAIN, forward) butterfly on chip in the level conv kernel
+FLAG_ABLATE_COLLAPSED_SYNTHESIS = 32  # (with FLAG_REFERENCE_CHAIN, forward) one closed-form synthesis pass
 ARITHMETIC_DTYPE = "f32"  # every kernel multiplies and accumulates in float32, whatever the storage type
 _DTYPES = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_NAMES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}

@@ -91,7 +91,7 @@ def test_scratch_memory_accounting(lib):
                  "convnext_s1_bf16", "convnext_s2_bf16", "convnext_s3_bf16", "convnext_s4_bf16"):
         wl = inputs.WORKLOADS[name]
         d = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wl.dtype)
-        assert wt.wtconv_plan_name(d) == "plane"
+        assert wt.wtconv_plan_name(d) in ("plane", "team")
         fb, bb = wt.wtconv_workspace_bytes(d)
         assert fb == 256 and bb < (8 << 20), (name, fb, bb)
     wl = inputs.WORKLOADS["large_f16"]
@@ -115,18 +115,21 @@ def test_host_planning_over_a_shape_sweep(lib):
                 for B, C in ((1, 1), (2, 3), (64, 96), (128, 768)):
                     d = wt.make_desc(B, C, H, W, 5, L, dt)
                     name = wt.wtconv_plan_name(d)
-                    assert name in ("plane", "tiled"), (H, W, L, dt, B, C, name)
+                    assert name in ("team", "plane", "tiled"), (H, W, L, dt, B, C, name)
                     seen.add(name)
                     nf, nb = wt.wtconv_launch_count(d)
-                    if name == "plane":
+                    if name == "team":
+                        assert nf == 1 and nb == 2
+                    elif name == "plane":
                         assert nf == 1 and nb in (2, 3)
                     else:
                         assert nf == L + 1 and nb == L + 2
+                    assert wt.wtconv_plan_describe(d).startswith(name)
                     fb, bb = wt.wtconv_workspace_bytes(d)
-                    assert fb >= (256 if name == "plane" else 0) and bb >= fb and bb > 0 and fb % 256 == 0 and bb % 256 == 0, (H, W, L, dt, B, C, fb, bb)
+                    assert fb >= (256 if name != "tiled" else 0) and bb >= fb and bb > 0 and fb % 256 == 0 and bb % 256 == 0, (H, W, L, dt, B, C, fb, bb)
                     for lvl in range(L + 1):
                         assert wt.wtconv_level_shape(d, lvl) == (-(-H // (1 << lvl)), -(-W // (1 << lvl)))
-    assert seen == {"plane", "tiled"}
+    assert seen == {"team", "plane", "tiled"}
 
 
 def test_binding_refuses_to_run_without_the_library(monkeypatch):

@@ -43,6 +43,31 @@ def test_small_fp32(wl, flags):
     assert_close(wl, run_gpu(wl, I, flags), run_oracle(wl, I))
 
 
+# Tiny planes with a channel count the team kernels can group (several planes per thread team); the same
+# shapes also run on the block-per-plane kernels (FLAG_NO_TEAM) and on the tiled path.
+TEAM_SHAPES = [
+    Workload("team_7x7", 5, 16, 7, 7, 5, 1, "f32", 51),
+    Workload("team_7x7_L2", 3, 8, 7, 7, 5, 2, "f32", 52),          # 7 -> 4 -> 2
+    Workload("team_8x8_L3", 2, 8, 8, 8, 5, 3, "f32", 53),          # grids shrink to 1 x 1
+    Workload("team_9x9_L2", 4, 4, 9, 9, 5, 2, "f32", 54),          # 9 -> 5 -> 3, odd at every level
+    Workload("team_5x10", 3, 8, 5, 10, 5, 1, "f32", 55),           # non-square
+    Workload("team_base_only", 2, 8, 6, 6, 5, 0, "f32", 56),
+    Workload("team_many_groups", 37, 24, 7, 7, 5, 1, "f32", 57),   # several channel groups per block, ragged unit ranges
+]
+TEAM_PATHS = [pytest.param(0, id="team"), pytest.param(wt.FLAG_NO_TEAM, id="plane"), pytest.param(wt.FLAG_TILED_ONLY, id="tiled")]
+
+
+@pytest.mark.parametrize("flags", TEAM_PATHS)
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("wl", TEAM_SHAPES, ids=lambda w: w.name)
+def test_tiny_planes(wl, dtype, flags):
+    wl = wl.with_(dtype=dtype)
+    I = inputs.make_inputs(wl, bias=True)
+    name = wt.wtconv_plan_name(wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, dtype, flags))
+    assert name == {0: "team", wt.FLAG_NO_TEAM: "plane", wt.FLAG_TILED_ONLY: "tiled"}[flags]
+    assert_close(wl, run_gpu(wl, I, flags), run_oracle(wl, I))
+
+
 @pytest.mark.parametrize("flags", PATHS)
 @pytest.mark.parametrize("wl", [SMALL[1], SMALL[4], SMALL[9]], ids=lambda w: w.name)
 def test_bias(wl, flags):
@@ -60,12 +85,13 @@ def test_small_16bit(wl, dtype, flags):
 
 
 @pytest.mark.parametrize("flags", PATHS)
-@pytest.mark.parametrize("shape", [(7, 7, 2), (29, 29, 4), (57, 33, 3), (56, 56, 3), (14, 14, 1), (28, 28, 2)])
+@pytest.mark.parametrize("shape", [(7, 7, 2), (29, 29, 4), (57, 33, 3), (56, 56, 3), (14, 14, 1), (28, 28, 2), (7, 7, 1, 8),
+                                   (9, 9, 3, 4)])
 def test_index_and_padding_math_bit_exact(shape, flags):
     """Dyadic inputs make every intermediate exact in fp32, so out and grad_x must equal the
     oracle bit for bit whatever the summation order; any difference is an index/sign/padding bug."""
-    H, W, L = shape
-    wl = Workload("dyadic", 2, 3, H, W, 5, L, "f32", 30)
+    H, W, L = shape[:3]
+    wl = Workload("dyadic", 2, shape[3] if len(shape) > 3 else 3, H, W, 5, L, "f32", 30)  # 8 / 4 channels: the team kernels' groups
     I = inputs.make_dyadic_inputs(wl, bias=True)
     out, gr = run_gpu(wl, I, flags)
     rout, rgr = run_oracle(wl, I)
