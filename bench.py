@@ -14,6 +14,9 @@ per GPU, k = 5: (C=96, 56x56, L=3), (C=192, 28x28, L=2), (C=384, 14x14, L=1), (C
   per_workload   every benchmark configuration (level sweep fp32/fp16, stage-1 fp32, the stage set, the
                  network's depth schedule, k = 3 / 7, the large planes) with forward / backward time,
                  elements/s, ALU and HBM fractions and the kernel family that served it (N = 1 only)
+  comparator     per level count L of the sweep: this library's own reference-style chain (separate operators,
+                 every intermediate in HBM, Sec. 3.1) timed beside the fused kernels, the cumulative ablation of
+                 Table 8 on the forward pass, and ncu DRAM bytes per element against Eq. 2 / Eq. 10 where captured
   cpu_baseline   the fp64 oracle on this machine's host cores on a bounded sample (rank 0, N = 1 only)
 
 `--workload NAME` times that single workload instead of the stage set (used for profiler captures).
@@ -42,14 +45,15 @@ TABLE = (["stage1_f32"] + ["sweep_L%d_f32" % l for l in range(1, 6)] + ["sweep_L
          STAGE_SET + ["convnext_s%d_bf16" % s for s in range(1, 5)] + ["stage1_k3_f32", "stage1_k7_f32"] +
          ["large_f16", "large_odd_f16"])
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (bytes; keyed by workload and kernel family).  Absent = no capture of that launch exists.
-NCU_DRAM_TRAFFIC = {}
-try:
-    with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as _f:
-        NCU_DRAM_TRAFFIC = {tuple(k.split("|")): v for k, v in json.load(_f).items() if not k.startswith("_")}
-except Exception:
-    pass
+# dram__bytes_read.sum + dram__bytes_write.sum per library call from the ncu captures summarised under profiles/
+# (bytes; keyed by workload and path).  Absent = no capture of that call exists.
+NCU_DRAM_TRAFFIC = {
+    # profiles/io_model_traffic_f32.md
+    ("traffic_L1_f32", "reference_fwd"): 4271524242, ("traffic_L1_f32", "tiled_fwd"): 1333854757,
+    ("traffic_L3_f32", "reference_fwd"): 5002461952, ("traffic_L3_f32", "tiled_fwd"): 1597085367,
+    ("traffic_L5_f32", "reference_fwd"): 5039999049, ("traffic_L5_f32", "tiled_fwd"): 1607475639,
+    ("sweep_L3_f32", "reference_fwd"): 948305810, ("sweep_L3_f32", "tiled_fwd"): 320324425, ("sweep_L3_f32", "plane_fwd"): 89365248,
+}
 
 
 def load_measured_peaks():
@@ -192,17 +196,19 @@ class Runner:
                 "training_step_peak": 4 * act + 2 * par + max(self.ws_fwd, self.ws_bwd)}
 
 
-def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions):
+def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions, direction="both"):
     """Regions of exactly K steps, repeated until `min_seconds` have been timed; every call is bracketed by events.
     Returns (region_ms list, per-runner [fwd_ms list, bwd_ms list])."""
     def step(i, ev=None):
         for j, r in enumerate(runners):
             if ev is not None:
                 ev[j][0].record(stream)
-            r.fwd(i, stream)
+            if direction != "bwd":
+                r.fwd(i, stream)
             if ev is not None:
                 ev[j][1].record(stream)
-            r.bwd(i, stream)
+            if direction != "fwd":
+                r.bwd(i, stream)
             if ev is not None:
                 ev[j][2].record(stream)
             all_reduce(r)
@@ -255,6 +261,68 @@ def row_for(r, fwd_ms, bwd_ms, peaks, io_model):
     }
 
 
+# Paper's own ratios on its hardware (RTX A6000, k = 5, geometric mean over its layer sweep), context only:
+# Table 2 (training step, reference / fused) and Table 3 (forward), fp32, L = 1..5.
+PAPER_TRAIN_RATIO_F32 = [3.71, 4.23, 4.34, 4.35, 4.33]
+PAPER_FWD_RATIO_F32 = [3.67, 4.20, 4.32, 4.35, 4.37]
+
+
+def comparator_rows(names, mk, wt, io_model, stream, torch, sync_all, have):
+    """Reference-style chain and ablation steps next to the fused kernels, one row per workload."""
+    REF, FA, CS = wt.FLAG_REFERENCE_CHAIN, wt.FLAG_ABLATE_FUSED_ANALYSIS, wt.FLAG_ABLATE_COLLAPSED_SYNTHESIS
+    med = statistics.median
+
+    def timed(fn, reps):
+        for i in range(2):
+            fn(i)
+        sync_all()
+        ts = []
+        for i in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); fn(i); e1.record(stream); sync_all()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return med(ts)
+
+    out = []
+    for name in names:
+        ours = have[name]
+        row = {"workload": name, "L": ours["L"], "storage": ours["storage"],
+               "fused_fwd_us": ours["fwd_us"], "fused_train_step_us": round(ours["fwd_us"] + ours["bwd_us"], 2)}
+        from paper_2608_10805_b200 import inputs
+        wl = inputs.WORKLOADS[name]
+        r = mk(wl, REF)
+        row["reference_fwd_us"] = round(timed(lambda i: r.fwd(i, stream), 5), 1)
+        row["reference_train_step_us"] = round(timed(lambda i: r.bwd(i, stream), 3), 1)  # this call = forward chain + backward chain
+        row["reference_launches"] = [r.nf, r.nb]
+        row["reference_workspace_bytes"] = [r.ws_fwd, r.ws_bwd]
+        del r
+        torch.cuda.empty_cache()
+        abl = {"reference": row["reference_fwd_us"]}
+        for label, fl in (("+fused_analysis", REF | FA), ("+collapsed_synthesis", REF | FA | CS), ("+scale_folding", wt.FLAG_TILED_ONLY)):
+            r = mk(wl, fl)
+            abl[label] = round(timed(lambda i: r.fwd(i, stream), 5), 1)
+            del r
+            torch.cuda.empty_cache()
+        abl["whole_plane_kernels"] = ours["fwd_us"]
+        row["ablation_fwd_us"] = abl
+        row["fwd_ratio_reference_over_fused"] = round(row["reference_fwd_us"] / ours["fwd_us"], 2)
+        row["train_ratio_reference_over_fused"] = round(row["reference_train_step_us"] / row["fused_train_step_us"], 2)
+        if ours["storage"] == "f32" and 1 <= ours["L"] <= 5:
+            row["paper_a6000_ratio"] = {"fwd": PAPER_FWD_RATIO_F32[ours["L"] - 1], "train": PAPER_TRAIN_RATIO_F32[ours["L"] - 1]}
+        n = wl.N
+        row["io_model_N"] = {"q_ref_fwd": round(io_model.q_ref(wl.L), 3), "q_fused_fwd": round(io_model.q_fused(wl.L), 3),
+                             "ours_fwd_compulsory": 2.0}
+        meas = {}
+        for kind in ("reference_fwd", "tiled_fwd", "plane_fwd", "plane_bwd"):
+            v = NCU_DRAM_TRAFFIC.get((name, kind))
+            if v is not None:
+                meas[kind] = round(v / (n * (4 if wl.dtype == "f32" else 2)), 3)
+        if meas:
+            row["ncu_dram_bytes_per_element_over_elem_size"] = meas
+        out.append(row)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -267,8 +335,11 @@ def main():
     ap.add_argument("--min-seconds", type=float, default=0.5, help="repeat the K-step region until this much is timed")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-table", action="store_true", help="skip the per_workload table")
+    ap.add_argument("--no-comparator", action="store_true", help="skip the reference-chain / ablation rows")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--tune", type=lambda s: int(s, 0), default=0, help="launch-plan override bits (see wtconv.h)")
+    ap.add_argument("--tune", type=lambda s: int(s, 0), default=0, help="desc.flags: path selection and launch-plan override bits (see wtconv.h)")
+    ap.add_argument("--direction", default="both", choices=["both", "fwd", "bwd"],
+                    help="profiler captures: enqueue only the forward or only the backward call of every step")
     args = ap.parse_args()
 
     from paper_2608_10805_b200 import inputs, io_model
@@ -310,14 +381,21 @@ def main():
     K, W = max(args.steps, 1), max(args.warmup, 3)
     for i in range(3):  # first calls: plan search, function attributes, module load
         for r in runners:
-            r.fwd(i, stream); r.bwd(i, stream)
+            if args.direction != "bwd":
+                r.fwd(i, stream)
+            if args.direction != "fwd":
+                r.bwd(i, stream)
     sync_all()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.2)
     t0 = time.time()
-    regions, fwd_ms, bwd_ms = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400)
+    regions, fwd_ms, bwd_ms = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400,
+                                           args.direction)
+    if args.direction != "both":  # a profiling run: the untimed call would divide by zero in the roofline rows
+        fwd_ms = [[max(v, 1e-6) for v in f] for f in fwd_ms]
+        bwd_ms = [[max(v, 1e-6) for v in b] for b in bwd_ms]
     t1 = time.time()
     med = statistics.median(regions)
     ms = torch.tensor([med], device=dev)
@@ -443,6 +521,18 @@ def main():
             del r
             torch.cuda.empty_cache()
         result["per_workload"] = table
+        if not args.no_comparator:
+            byname = {r_["workload"]: r_ for r_ in table}
+            result["io_model_validation"] = [
+                {"workload": w_, "N": inputs.WORKLOADS[w_].N, "L": inputs.WORKLOADS[w_].L,
+                 "ncu_dram_over_4N": {k_: round(NCU_DRAM_TRAFFIC[(w_, k_)] / (4.0 * inputs.WORKLOADS[w_].N), 3)
+                                      for k_ in ("reference_fwd", "tiled_fwd") if (w_, k_) in NCU_DRAM_TRAFFIC},
+                 "model": {"q_ref": round(io_model.q_ref(inputs.WORKLOADS[w_].L), 3),
+                           "q_fused_minus_base_pass": round(io_model.q_fused(inputs.WORKLOADS[w_].L) - 2.0, 3)},
+                 "source": "profiles/io_model_traffic_f32.md"}
+                for w_ in ("traffic_L1_f32", "traffic_L3_f32", "traffic_L5_f32")]
+            result["comparator"] = comparator_rows(["sweep_L%d_f32" % l for l in range(1, 6)] + ["sweep_L3_f16", "stage1_f32"],
+                                                   mk, wt, io_model, stream, torch, sync_all, byname)
     print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()

@@ -184,7 +184,9 @@ wtconv_status wtconv_read_status(const wtconv_desc *desc, const void *workspace,
  *     device current); make that first call outside any stream capture.  Later calls on that device reuse it.
  *   - All calls on one device share the one array, and it keeps whatever the last call left in it.  Each call
  *     clears what has to start at zero, so stale contents are harmless, but two calls whose kernels overlap
- *     on the GPU (different streams) race on it: serialise them, or use wtconv_backward with two workspaces. */
+ *     on the GPU (different streams) race on it: serialise them, or use wtconv_backward with two workspaces.
+ *   - The kernels' status word lives in the array too: read it with wtconv_read_status(desc, NULL, ...).
+ *   - WTCONV_ERR_ARCH (device is not compute capability 10.x) is reported before the array is looked up. */
 #define WTCONV_STATIC_SCRATCH_BYTES (8u << 20)
 wtconv_status wtconv_backward_static(const wtconv_desc *desc, const void *x, const void *grad_out,
                                      const float *w0, const float *s0, const float *b0,

@@ -234,23 +234,25 @@ static __global__ void bias_grads_kernel(const float *__restrict__ sumg, const f
 static __global__ void fill_kernel(float *__restrict__ p, float v, size_t n) {
     for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) p[e] = v;
 }
-// out = Q + sum_l (Proposition 2 term of U^l): the collapsed synthesis of the ablation, one pass over the output
+// out = Q + sum_l (Proposition 2 term of U^l): the collapsed synthesis of the ablation, one pass over the output;
+// a 4 x 4 pixel block per thread, 64 x 64 pixel tiles per block (the layout of the fused synthesis kernel)
 template <typename T>
-__global__ void closed_form_add_kernel(const float *__restrict__ Q, int H, int W, int L, tiled::LevelPtrs lv, size_t P, T *__restrict__ out) {
-    const size_t HW = (size_t)H * W, n = P * HW;
-    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
-        const size_t p = e / HW;
-        const int r = (int)(e - p * HW), y = r / W, x = r - y * W;
-        float v = Q[e], scale = 1.f;
-        for (int l = 1; l <= L; ++l) {
-            scale *= 0.5f;
-            const int Wl = lv.Wl[l - 1];
-            const size_t S = (size_t)lv.Hl[l - 1] * Wl;
-            const float *z = lv.z[l - 1] + p * 4 * S + (size_t)(y >> l) * Wl + (x >> l);
-            v += synth_term(z[0], z[S], z[2 * S], z[3 * S], (y >> (l - 1)) & 1, (x >> (l - 1)) & 1, scale);
-        }
-        stf(out + e, v);
-    }
+__global__ void __launch_bounds__(tiled::NTHREADS)
+closed_form_add_kernel(const float *__restrict__ Q, int H, int W, int L, tiled::LevelPtrs lv, T *__restrict__ out) {
+    const int ntx = tiled::tiles_of(W, tiled::STW), ntile = ntx * tiled::tiles_of(H, tiled::STH);
+    const size_t p = blockIdx.x / ntile;
+    const int tile = (int)(blockIdx.x - p * ntile);
+    const int X0 = (tile % ntx) * tiled::STW + 4 * (threadIdx.x & 15), Y0 = (tile / ntx) * tiled::STH + 4 * (threadIdx.x >> 4);
+    if (X0 >= W || Y0 >= H) return;
+    const tiled::Z12 z = tiled::load_z12(lv, L, p, Y0, X0);
+    float a[4][4];
+    const float *q = Q + p * H * W;
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) a[r][c] = (Y0 + r < H && X0 + c < W) ? __ldg(q + (size_t)(Y0 + r) * W + X0 + c) : 0.f;
+    tiled::block_synthesis(lv, L, p, Y0, X0, z, a);
+    tiled::store_block<T>(out + p * H * W, H, W, Y0, X0, a);
 }
 
 // ---------------------------------------------------------------- workspace plan
@@ -336,7 +338,7 @@ wtconv_status forward(const wtconv_desc *d, const T *x, const float *w0, const f
         // one pass: Proposition 2 over all U^l plus the base result, straight into out
         tiled::LevelPtrs lv = {};
         for (int l = 1; l <= L; ++l) { lv.z[l - 1] = F(pl.U[l - 1]); lv.Hl[l - 1] = pl.sh.Hs[l]; lv.Wl[l - 1] = pl.sh.Ws[l]; }
-        closed_form_add_kernel<T><<<nblk(pl.N), RT, 0, st>>>(F(pl.Qb), d->H, d->W, L, lv, P, out);
+        closed_form_add_kernel<T><<<nb0, tiled::NTHREADS, 0, st>>>(F(pl.Qb), d->H, d->W, L, lv, out);
     } else {
         for (int l = L; l >= 1; --l) {
             const int Hp = pl.sh.Hs[l - 1], Wp = pl.sh.Ws[l - 1], Hl = pl.sh.Hs[l], Wl = pl.sh.Ws[l];

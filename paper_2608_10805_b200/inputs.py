@@ -53,6 +53,9 @@ WORKLOADS = {
     # kernel-size variants of the stage-1 layer
     "stage1_k3_f32": Workload("stage1_k3_f32", 16, 96, 56, 56, 3, 3, "f32", 6),
     "stage1_k7_f32": Workload("stage1_k7_f32", 16, 96, 56, 56, 7, 3, "f32", 6),
+    # the paper's traffic-validation shape (C = 128, 128 x 128, k = 5) at a batch that makes one tensor (268 MB) larger
+    # than the 126 MB L2, so that DRAM counters see what the I/O model counts
+    **{"traffic_L%d_f32" % L: Workload("traffic_L%d_f32" % L, 32, 128, 128, 128, 5, L, "f32", 7) for L in (1, 3, 5)},
     "large_f16": Workload("large_f16", 16, 256, 256, 256, 5, 5, "f16", 4),
     "large_odd_f16": Workload("large_odd_f16", 16, 256, 225, 225, 5, 5, "f16", 4),
 }

@@ -132,6 +132,30 @@ def test_host_planning_over_a_shape_sweep(lib):
     assert seen == {"team", "plane", "tiled"}
 
 
+def test_host_step_workspace_covers_its_batch_chunks(lib):
+    """wtconv_step_host runs the kernels chunk by chunk on B / n images (n up to 8); the scratch a chunk needs is not
+    monotone in B (the gradient partial slots depend on how blocks split the units), so the reported size must
+    cover the chunk descriptor as well as the whole batch."""
+    from paper_2608_10805_b200 import inputs
+    shapes = [(96, 56, 56, 3), (192, 28, 28, 2), (384, 14, 14, 1), (768, 7, 7, 1), (512, 7, 7, 1), (128, 64, 64, 3)]
+    for C, H, W, L in shapes:
+        for dt, esz in (("f32", 4), ("bf16", 2)):
+            for B in (8, 16, 32, 64, 96, 128, 192, 256, 384):
+                d = wt.make_desc(B, C, H, W, 5, L, dt)
+                total = wt.wtconv_step_host_workspace_bytes(d)
+                act = -(-B * C * H * W * esz // 256) * 256
+                par = sum(-(-n * 4 // 256) * 256 for n in (C * 25, C, C, L * C * 100, L * C * 4))
+                scratch = total - 4 * act - 10 * par
+                per_image = C * H * W * esz
+                for n in (8, 4, 2):  # the library's chunking rule
+                    if B % n == 0 and B // n >= 4 and (B // n * per_image) % 16 == 0 and B // n * per_image >= (4 << 20):
+                        fb, bb = wt.wtconv_workspace_bytes(wt.make_desc(B // n, C, H, W, 5, L, dt))
+                        assert max(fb, bb) <= scratch, (C, H, W, L, dt, B, n, max(fb, bb), scratch)
+                        break
+                fb, bb = wt.wtconv_workspace_bytes(d)
+                assert max(fb, bb) <= scratch
+
+
 def test_binding_refuses_to_run_without_the_library(monkeypatch):
     monkeypatch.setattr(wt, "_lib", None)
     monkeypatch.setattr(wt, "LIB_PATH", "/nonexistent/libwtconv_b200.so")

@@ -7,13 +7,14 @@ from paper_2608_10805_b200 import inputs
 from paper_2608_10805_b200 import wtconv as wt
 from paper_2608_10805_b200.inputs import Workload
 
-from helpers import to_dev
+from helpers import TOL, rel_err, to_dev
+from oracle import wtconv_oracle as O
 
 pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("wl", [
-    Workload("graph_stage4", 4, 16, 7, 7, 5, 2, "bf16", 41),     # plane path, fused backward
+    Workload("graph_stage4", 4, 16, 7, 7, 5, 2, "bf16", 41),     # team kernels
     Workload("graph_stage2", 2, 8, 28, 28, 5, 2, "f32", 42),
     Workload("graph_tiled", 1, 3, 90, 75, 5, 3, "f32", 43),      # tiled path (several launches per call)
 ], ids=lambda w: w.name)
@@ -55,5 +56,11 @@ def test_step_replays_from_a_cuda_graph(wl):
         assert torch.equal(got, want)  # same kernels, same order: bit-identical (the reductions are fixed-order)
     x.copy_(to_dev(I2["x"], tdt)); g.copy_(to_dev(I2["g"], tdt))
     graph.replay()
-    for got, want in zip(snapshot(), eager2):
+    replayed = snapshot()
+    for got, want in zip(replayed, eager2):
         assert torch.equal(got, want)
+    # and the replayed step is the operator itself: every tensor against the fp64 oracle on the second input set
+    ref_out = O.forward(I2["x"], I1["w0"], I1["s0"], None, I1["wl"], I1["sl"], wl.L)
+    ref = O.backward(I2["x"], I2["g"], I1["w0"], I1["s0"], None, I1["wl"], I1["sl"], wl.L)
+    for got, want in zip(replayed, (ref_out, ref["dx"], ref["dw0"], ref["ds0"], ref["dwl"], ref["dsl"])):
+        assert rel_err(got.double().cpu().numpy(), want) <= TOL[wl.dtype]
