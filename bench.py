@@ -52,6 +52,12 @@ NCU_DRAM_TRAFFIC = {
     ("traffic_L1_f32", "reference_fwd"): 4271524242, ("traffic_L1_f32", "tiled_fwd"): 1333854757,
     ("traffic_L3_f32", "reference_fwd"): 5002461952, ("traffic_L3_f32", "tiled_fwd"): 1597085367,
     ("traffic_L5_f32", "reference_fwd"): 5039999049, ("traffic_L5_f32", "tiled_fwd"): 1607475639,
+    # profiles/plane_kernels_stage_set_bf16_sections.md (kernel + epilogue of one call)
+    ("stage1_bf16", "plane_fwd"): 104200000, ("stage1_bf16", "plane_bwd"): 201700000,
+    # profiles/large_planes_traffic.md
+    ("large_f16", "window_fwd"): 1797000000, ("large_f16", "window_bwd"): 3089000000,
+    ("large_f16", "tiled_fwd"): 4988000000, ("large_f16", "tiled_bwd"): 7101000000,
+    ("large_odd_f16", "window_fwd"): 1387000000, ("large_odd_f16", "window_bwd"): 2383000000,
     ("sweep_L3_f32", "reference_fwd"): 948305810, ("sweep_L3_f32", "tiled_fwd"): 320324425, ("sweep_L3_f32", "plane_fwd"): 89365248,
 }
 
@@ -256,6 +262,8 @@ def row_for(r, fwd_ms, bwd_ms, peaks, io_model):
         "bound": "alu" if alu_floor >= hbm_floor else "hbm",
         "roof_frac": round(max(alu_floor, hbm_floor) / t_s, 4),
         "workspace_bytes": [r.ws_fwd, r.ws_bwd],
+        "ncu_dram_bytes": {k_[1]: v_ for k_, v_ in NCU_DRAM_TRAFFIC.items() if k_[0] == wl.name} or None,
+        "compulsory_bytes": [by_f, by_s - by_f],
         "paper_q_fused_fwd_N": round(io_model.q_fused(wl.L), 3) if wl.L else None,
         "paper_q_ref_fwd_N": round(io_model.q_ref(wl.L), 3) if wl.L else None,
     }
@@ -456,15 +464,21 @@ def main():
     by_step = sum(io_model.compulsory_bytes(r.wl.N, r.esz, "fwd+bwd") for r in runners)
     alu_floor_ms = fl_step / (FP32_ALU_PEAK_TFLOPS * 1e12) * 1e3
     hbm_floor_ms = by_step / (peaks["hbm_gbs"] * 1e9) * 1e3
-    # roofline: the stage furthest below its roof, and of its two calls the longer one
-    worst = min(range(len(rows)), key=lambda j: rows[j]["roof_frac"])
-    wr, wrow = runners[worst], rows[worst]
-    fl_f = io_model.algorithmic_flops(wr.wl.B, wr.wl.C, wr.wl.H, wr.wl.W, wr.wl.k, wr.wl.L, "fwd")
-    if wrow["bwd_us"] >= wrow["fwd_us"]:
-        dom_kind, dom_ms, dom_fl = "backward", mean(bwd_ms[worst]), 2 * fl_f
-    else:
-        dom_kind, dom_ms, dom_fl = "forward", mean(fwd_ms[worst]), fl_f
-    achieved = dom_fl / (dom_ms * 1e-3) / 1e12
+    # roofline: the dominant kernel = the library call with the largest share of the step time; the call furthest below
+    # its roof is reported beside it (roofline_worst_call)
+    def call_entry(j, kind):
+        r_, row_ = runners[j], rows[j]
+        f_ = io_model.algorithmic_flops(r_.wl.B, r_.wl.C, r_.wl.H, r_.wl.W, r_.wl.k, r_.wl.L, "fwd")
+        ms_, fl_ = (mean(bwd_ms[j]), 2 * f_) if kind == "backward" else (mean(fwd_ms[j]), f_)
+        ach_ = fl_ / (ms_ * 1e-3) / 1e12
+        return {"bound": row_["bound"], "kernel": "%s call of %s (%s kernels)" % (kind, r_.wl.name, r_.plan),
+                "achieved": ach_, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": ach_ / FP32_ALU_PEAK_TFLOPS,
+                "traffic": NCU_DRAM_TRAFFIC.get((r_.wl.name, "plane_bwd" if kind == "backward" else "plane_fwd")),
+                "peak_source": PEAK_SOURCE, "launch_ms": ms_, "flops_per_launch": fl_,
+                "share_of_step": ms_ / (sum(mean(v) for v in fwd_ms) + sum(mean(v) for v in bwd_ms))}
+    calls = [call_entry(j, kind) for j in range(len(rows)) for kind in ("forward", "backward")]
+    dominant = max(calls, key=lambda c_: c_["launch_ms"])
+    worst_call = min(calls, key=lambda c_: c_["frac"])
     result = {
         "metric": "wtconv_fwd_bwd_elements_per_s", "value": value, "unit": "elements/s", "n_gpus": world,
         "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True,
@@ -482,11 +496,10 @@ def main():
         "region_ms": {"min": min(regions), "median": med, "max": max(regions), "n": len(regions)},
         "e2e": e2e,
         "gpu_launches": sum(r.nf + r.nb for r in runners) * K,
-        "roofline": {"bound": wrow["bound"], "kernel": "%s call of %s (%s kernels)" % (dom_kind, wr.wl.name, wr.plan),
-                     "achieved": achieved, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s",
-                     "frac": achieved / FP32_ALU_PEAK_TFLOPS,
-                     "traffic": NCU_DRAM_TRAFFIC.get((wr.wl.name, dom_kind)),
-                     "peak_source": PEAK_SOURCE, "launch_ms": dom_ms, "flops_per_launch": dom_fl},
+        "roofline": dominant,
+        "roofline_worst_call": worst_call,
+        "roofline_calls": [{"kernel": c_["kernel"], "launch_ms": round(c_["launch_ms"], 4), "frac": round(c_["frac"], 4),
+                            "share_of_step": round(c_["share_of_step"], 4)} for c_ in calls],
         "step_rooflines": {
             "alu_frac": alu_floor_ms / ms_step,
             "hbm_compulsory_gbs": by_step / (ms_step * 1e-3) / 1e9,

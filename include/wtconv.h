@@ -77,6 +77,11 @@ typedef enum {
  * normally with nothing in flight (outputs are then invalid by design).  Never set it in production. */
 #define WTCONV_FLAG_TEST_NO_COPY 2u
 #define WTCONV_FLAG_NO_TEAM 4u /* never take the team kernels for small planes (used to test the block-per-plane kernels on them) */
+#define WTCONV_FLAG_NO_WINDOW 64u /* never take the window kernels for large planes (used to test the tiled path on them) */
+/* Large planes are served by the window kernels (levels 1-2 on chip, about 2.2 N elements of HBM traffic) when their
+ * rows are not 16-byte multiples, and by the tiled kernels (per-level launches, Q_fused - 2 N of traffic, but faster
+ * on this GPU when rows are aligned) otherwise; this flag takes the window kernels wherever they apply. */
+#define WTCONV_FLAG_PREFER_WINDOW 128u
 /* Comparator: run the layer as the chain of separate operators of Sec. 3.1 (analysis, depthwise conv, scale pass,
  * slice, add, concatenate, synthesis per level; base conv, scale pass, add), every intermediate in HBM, as plain
  * kernels of this library.  It is what the paper measures its fused kernels against (Eq. 2 vs Eq. 10, Tables 1-3);
@@ -124,7 +129,8 @@ wtconv_status wtconv_level_shape(const wtconv_desc *desc, int level, int32_t *Hl
 wtconv_status wtconv_workspace_bytes(const wtconv_desc *desc, size_t *fwd_bytes, size_t *bwd_bytes);
 
 /* Name of the kernel family a descriptor dispatches to ("team" = small planes, several per thread team; "plane" =
- * one block per whole plane in shared memory; "tiled" = per-level tiled kernels).  Host call; returns NULL for
+ * one block per whole plane in shared memory; "window" = large planes cut into windows with levels 1-2 on chip;
+ * "tiled" = per-level tiled kernels; "reference-chain" = the comparator).  Host call; returns NULL for
  * an invalid desc. */
 const char *wtconv_plan_name(const wtconv_desc *desc);
 

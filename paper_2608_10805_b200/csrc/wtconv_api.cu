@@ -7,6 +7,7 @@
 #include "tiled_kernels.cuh"
 #include "plane_kernels.cuh"
 #include "team_kernels.cuh"
+#include "window_kernels.cuh"
 #include "tiled_host.cuh"
 #include "reference_chain.cuh"
 
@@ -23,6 +24,11 @@ WT_TEAM_INSTANTIATE(float, extern)
 WT_TEAM_INSTANTIATE(__half, extern)
 WT_TEAM_INSTANTIATE(__nv_bfloat16, extern)
 }  // namespace team
+namespace window {
+WT_WINDOW_INSTANTIATE(float, extern)
+WT_WINDOW_INSTANTIATE(__half, extern)
+WT_WINDOW_INSTANTIATE(__nv_bfloat16, extern)
+}  // namespace window
 namespace host {
 WT_TILED_INSTANTIATE(float, 3, extern)
 WT_TILED_INSTANTIATE(float, 5, extern)
@@ -87,6 +93,17 @@ bool use_plane_path(const wtconv_desc *d) {  // any kernel family that keeps who
     return use_team_path(d) || wt::plane::supported(d->H, d->W, d->k, d->L, d->dtype);
 }
 
+// Large planes (k = 5): windows with levels 1-2 on chip, deeper levels on the whole-plane kernels over a carrier.
+bool use_window_path(const wtconv_desc *d) {
+    if (d->flags & (WTCONV_FLAG_TILED_ONLY | WTCONV_FLAG_NO_WINDOW | WTCONV_FLAG_REFERENCE_CHAIN)) return false;
+    if (d->flags >> 8) return false;
+    if (use_plane_path(d)) return false;
+    // Measured on B200: with 16-byte aligned rows the per-level tiled kernels are as fast or faster (they stream whole
+    // rows), with unaligned rows (225-wide 16-bit planes) they fall to element loads and the window kernels win.
+    if (((size_t)d->W * elem_bytes(d->dtype)) % 16 == 0 && !(d->flags & WTCONV_FLAG_PREFER_WINDOW)) return false;
+    return wt::window::supported(d->B, d->C, d->H, d->W, d->k, d->L, d->dtype);
+}
+
 template <typename T, int K>
 wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, const float *s0, const float *b0,
                          const float *wl, const float *sl, void *out, char *ws, cudaStream_t st) {
@@ -95,6 +112,12 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
         if (use_team_path(d))
             return wt::team::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st,
                                         (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, team_force_g(d)) == cudaSuccess
+                       ? WTCONV_OK
+                       : WTCONV_ERR_CUDA;
+    }
+    if constexpr (K == 5) {
+        if (use_window_path(d))
+            return wt::window::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
@@ -120,6 +143,15 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
             wt::EpiloguePtrs ep = {};
             if (wt::team::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl, (T *)gx,
                                       ws, &ep, st, (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, team_force_g(d)) != cudaSuccess)
+                return WTCONV_ERR_CUDA;
+            return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
+        }
+    }
+    if constexpr (K == 5) {
+        if (use_window_path(d)) {
+            wt::EpiloguePtrs ep = {};
+            if (wt::window::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl, (T *)gx, ws, &ep,
+                                        st) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
         }
@@ -157,11 +189,13 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
 size_t fwd_ws_bytes(const wtconv_desc *d) {
     if (use_ref_chain(d)) return wt::refchain::make_plan(d).fwd_bytes;
     if (use_plane_path(d)) return align_up(wt::plane::forward_workspace_bytes(d->B, d->C, d->H, d->W, d->L));
+    if (use_window_path(d)) return align_up(wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).fwd_bytes);
     return make_tiled_plan(d).fwd_bytes;
 }
 size_t bwd_ws_bytes(const wtconv_desc *d) {
     if (use_ref_chain(d)) return wt::refchain::make_plan(d).bwd_bytes;
     if (use_team_path(d)) return align_up(wt::team::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), team_force_g(d)));
+    if (use_window_path(d)) return align_up(wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).bwd_bytes);
     if (use_plane_path(d)) return align_up(wt::plane::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), d->flags >> 8));
     return make_tiled_plan(d).bwd_bytes;
 }
@@ -291,7 +325,7 @@ wtconv_status wtconv_workspace_bytes(const wtconv_desc *d, size_t *fwd_bytes, si
 
 const char *wtconv_plan_name(const wtconv_desc *d) {
     if (validate_desc(d) != WTCONV_OK) return nullptr;
-    return use_ref_chain(d) ? "reference-chain" : use_team_path(d) ? "team" : use_plane_path(d) ? "plane" : "tiled";
+    return use_ref_chain(d) ? "reference-chain" : use_team_path(d) ? "team" : use_plane_path(d) ? "plane" : use_window_path(d) ? "window" : "tiled";
 }
 
 wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
@@ -305,7 +339,14 @@ wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
                  (d->flags & WTCONV_FLAG_ABLATE_COLLAPSED_SYNTHESIS) ? " +collapsed-synthesis" : "");
     else if (use_team_path(d))
         wt::team::describe(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), buf, n, team_force_g(d));
-    else if (use_plane_path(d))
+    else if (use_window_path(d)) {
+        wt::window::WGeom wf, wb;
+        wt::window::make_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), false, wf);
+        wt::window::make_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), true, wb);
+        snprintf(buf, n, "window fwd[%dx%d px, %d thr x %d/SM, buffers=%d, %s] bwd[%dx%d px, %d thr x %d/SM, buffers=%d, np=%d]%s",
+                 wf.WH, wf.WW, wf.g.nthreads, wf.g.blocks_per_sm, wf.nbuf, wf.aligned ? "aligned rows" : "unaligned rows", wb.WH, wb.WW,
+                 wb.g.nthreads, wb.g.blocks_per_sm, wb.nbuf, wb.g.np, d->L > 2 ? " + whole-plane kernels on the level-2 carrier" : "");
+    } else if (use_plane_path(d))
         wt::plane::describe(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), d->flags >> 8, buf, n);
     else
         snprintf(buf, n, "tiled fwd[%d launches] bwd[%d launches]", d->L + 1, d->L + 2);
@@ -320,6 +361,10 @@ wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *b
         const int nf = (fa ? 1 : 0) + d->L * (fa ? 2 : 3) + (d->L > 1 && !fa ? d->L - 1 : 0) + 2 + (cs ? 1 : 2 * d->L + 1);
         if (fwd) *fwd = nf;
         if (bwd) *bwd = (4 * d->L + 3) + 7 + 9 * d->L;  // plain forward chain + gradient launches (approximate for L > 1 slices)
+    } else if (use_window_path(d)) {
+        // window kernel (+ carrier, scale fill and the whole-plane kernel when L > 2); backward: + second carrier, epilogue
+        if (fwd) *fwd = d->L > 2 ? 4 : 1;
+        if (bwd) *bwd = d->L > 2 ? 7 : 2;
     } else if (use_team_path(d)) {
         if (fwd) *fwd = 1;
         if (bwd) *bwd = 2;  // fused backward + epilogue (plus one memset node)
@@ -554,7 +599,9 @@ wtconv_status wtconv_read_status(const wtconv_desc *d, const void *workspace, in
         workspace = scratch;
     }
     if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
-    if (!use_plane_path(d)) {  // the tiled kernels wait for nothing and keep no status word
+    if (use_window_path(d) && d->L > 2)  // the carrier's whole-plane kernels keep the only status word of this path
+        workspace = (const char *)workspace + wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).deep;
+    else if (!use_plane_path(d)) {  // the tiled, window (L <= 2) and reference kernels wait for nothing and keep no status word
         *h_flag = 0;
         return WTCONV_OK;
     }

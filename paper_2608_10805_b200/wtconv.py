@@ -17,6 +17,8 @@ F32, F16, BF16 = 0, 1, 2
 FLAG_TILED_ONLY = 1
 FLAG_TEST_NO_COPY = 2
 FLAG_NO_TEAM = 4
+FLAG_NO_WINDOW = 64
+FLAG_PREFER_WINDOW = 128
 FLAG_REFERENCE_CHAIN = 8            # comparator: the layer as separate operators with every intermediate in HBM
 FLAG_ABLATE_FUSED_ANALYSIS = 16     # (with FLAG_REFERENCE_CHAIN, forward) butterfly on chip in the level conv kernel
 FLAG_ABLATE_COLLAPSED_SYNTHESIS = 32  # (with FLAG_REFERENCE_CHAIN, forward) one closed-form synthesis pass

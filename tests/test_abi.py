@@ -74,11 +74,18 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
 
 
 def test_plan_and_launch_count(lib):
-    d = wt.make_desc(2, 3, 300, 300, 5, 3, "f32")
-    assert wt.wtconv_plan_name(d) == "tiled"
-    assert wt.wtconv_launch_count(d) == (4, 5)
+    d = wt.make_desc(2, 3, 301, 301, 5, 3, "f32")  # rows that are not 16-byte multiples: window kernels
+    assert wt.wtconv_plan_name(d) == "window"
+    assert wt.wtconv_launch_count(d) == (4, 7)
+    assert wt.wtconv_launch_count(wt.make_desc(2, 3, 301, 301, 5, 2, "f32")) == (1, 2)
+    assert wt.wtconv_plan_name(wt.make_desc(2, 3, 300, 300, 5, 3, "f32")) == "tiled"
+    assert wt.wtconv_plan_name(wt.make_desc(2, 3, 300, 300, 5, 3, "f32", wt.FLAG_PREFER_WINDOW)) == "window"
+    dn = wt.make_desc(2, 3, 300, 300, 5, 3, "f32", wt.FLAG_NO_WINDOW)
+    assert wt.wtconv_plan_name(dn) == "tiled"
+    assert wt.wtconv_launch_count(dn) == (4, 5)
     dt = wt.make_desc(2, 3, 56, 56, 5, 3, "f32", wt.FLAG_TILED_ONLY)
     assert wt.wtconv_plan_name(dt) == "tiled"
+    assert wt.wtconv_plan_name(wt.make_desc(2, 3, 56, 56, 7, 3, "f32")) == "tiled"  # k = 3 / 7: tiled kernels
 
 
 def test_scratch_memory_accounting(lib):
@@ -95,7 +102,12 @@ def test_scratch_memory_accounting(lib):
         fb, bb = wt.wtconv_workspace_bytes(d)
         assert fb == 256 and bb < (8 << 20), (name, fb, bb)
     wl = inputs.WORKLOADS["large_f16"]
-    d = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wl.dtype)
+    d = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wl.dtype, wt.FLAG_PREFER_WINDOW)
+    assert wt.wtconv_plan_name(d) == "window"
+    fb, bb = wt.wtconv_workspace_bytes(d)
+    n16 = wl.N // 16 * 4  # one fp32 carrier-sized tensor (a sixteenth of the elements)
+    assert 3 * n16 <= fb <= 3 * n16 + (8 << 20) and fb <= bb <= 3 * n16 + (16 << 20)  # X2, R3, G2: 0.75 B per element
+    d = wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wl.dtype, wt.FLAG_NO_WINDOW)
     fb, _ = wt.wtconv_workspace_bytes(d)
     P, coeffs = wl.B * wl.C, 0
     for l in range(1, wl.L + 1):
@@ -115,13 +127,15 @@ def test_host_planning_over_a_shape_sweep(lib):
                 for B, C in ((1, 1), (2, 3), (64, 96), (128, 768)):
                     d = wt.make_desc(B, C, H, W, 5, L, dt)
                     name = wt.wtconv_plan_name(d)
-                    assert name in ("team", "plane", "tiled"), (H, W, L, dt, B, C, name)
+                    assert name in ("team", "plane", "window", "tiled"), (H, W, L, dt, B, C, name)
                     seen.add(name)
                     nf, nb = wt.wtconv_launch_count(d)
                     if name == "team":
                         assert nf == 1 and nb == 2
                     elif name == "plane":
                         assert nf == 1 and nb in (2, 3)
+                    elif name == "window":
+                        assert (nf, nb) == ((4, 7) if L > 2 else (1, 2))
                     else:
                         assert nf == L + 1 and nb == L + 2
                     assert wt.wtconv_plan_describe(d).startswith(name)
@@ -129,7 +143,7 @@ def test_host_planning_over_a_shape_sweep(lib):
                     assert fb >= (256 if name != "tiled" else 0) and bb >= fb and bb > 0 and fb % 256 == 0 and bb % 256 == 0, (H, W, L, dt, B, C, fb, bb)
                     for lvl in range(L + 1):
                         assert wt.wtconv_level_shape(d, lvl) == (-(-H // (1 << lvl)), -(-W // (1 << lvl)))
-    assert seen == {"team", "plane", "tiled"}
+    assert seen == {"team", "plane", "window", "tiled"}
 
 
 def test_host_step_workspace_covers_its_batch_chunks(lib):
