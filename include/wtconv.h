@@ -96,7 +96,8 @@ typedef enum {
 /* Launch-plan overrides for the plane-resident kernels, for tuning experiments (0 = let the planner choose):
  *   bits  8-12  threads per block / 32 of the forward / input-gradient kernel
  *   bits 13-15  resident blocks per SM of that kernel
- *   bits 16-21  planes per work unit of that kernel
+ *   bits 16-21  planes per work unit of that kernel (the only override the team kernels for tiny planes honour:
+ *               planes per team unit, forward and backward)
  *   bits 22-27  planes per work unit of the backward kernels
  *   bit  28     never prefetch with bulk copies      bit 29  never use the fused backward kernel
  *   bit  30     only 4 x 8 register tiles            bit 31  only 4 x 4 register tiles

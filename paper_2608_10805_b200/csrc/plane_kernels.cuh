@@ -94,7 +94,9 @@ __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ------------------------------------------------------------------ geometry (host-planned, passed by value)
-// Division by a launch-invariant divisor as multiply-high: exact while dividend * divisor < 2^32.
+// Division by a launch-invariant divisor as multiply-high: exact while dividend * divisor < 2^32.  Every use divides
+// an index inside one work unit (tiles, staging patches or coefficients of at most 64 planes: below 2^18) by a
+// per-plane count (below 2^13); indices over the whole tensor (units, images) are never divided this way.
 struct FastDiv {
     unsigned mul, d;
 };
