@@ -202,8 +202,11 @@ class Runner:
                 "training_step_peak": 4 * act + 2 * par + max(self.ws_fwd, self.ws_bwd)}
 
 
-def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions, direction="both"):
-    """Regions of exactly K steps, repeated until `min_seconds` have been timed; every call is bracketed by events.
+def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions, direction="both",
+                 per_call=True):
+    """Regions of exactly K steps, repeated until `min_seconds` have been timed.  per_call: every library call is
+    bracketed by events as well (an event between two kernels keeps the second from starting behind the tail of the
+    first, so regions timed this way run a little longer than a plain sequence of calls).
     Returns (region_ms list, per-runner [fwd_ms list, bwd_ms list])."""
     def step(i, ev=None):
         for j, r in enumerate(runners):
@@ -224,7 +227,8 @@ def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_se
     regions, fwd, bwd = [], [[] for _ in runners], [[] for _ in runners]
     total = 0.0
     while len(regions) < max_regions and (total < min_seconds or not regions):
-        evs = [[tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in runners] for _ in range(K)]
+        evs = [[tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in runners] if per_call else None
+               for _ in range(K)]
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         sync_all()
         e0.record(stream)
@@ -235,7 +239,7 @@ def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_se
         ms = e0.elapsed_time(e1)
         regions.append(ms)
         total += ms * 1e-3
-        for ev in evs:
+        for ev in evs if per_call else []:
             for j in range(len(runners)):
                 fwd[j].append(ev[j][0].elapsed_time(ev[j][1]))
                 bwd[j].append(ev[j][1].elapsed_time(ev[j][2]))
@@ -399,8 +403,12 @@ def main():
         sampler.start()
         time.sleep(0.2)
     t0 = time.time()
-    regions, fwd_ms, bwd_ms = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400,
-                                           args.direction)
+    # the headline: plain sequences of calls, nothing between them on the stream
+    regions, _, _ = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400, args.direction,
+                                 per_call=False)
+    # the per-call split behind the roofline entries: the same steps with an event around every call
+    call_regions, fwd_ms, bwd_ms = time_regions(runners, K, 0, stream, torch, sync_all, all_reduce, 0.1 if args.min_seconds else 0.0,
+                                                50, args.direction)
     if args.direction != "both":  # a profiling run: the untimed call would divide by zero in the roofline rows
         fwd_ms = [[max(v, 1e-6) for v in f] for f in fwd_ms]
         bwd_ms = [[max(v, 1e-6) for v in b] for b in bwd_ms]
@@ -488,8 +496,10 @@ def main():
                                "L": r.wl.L, "storage_dtype": r.wl.dtype, "plan": r.plan} for r in runners],
                    "l2": "a step touches %d MB (> 126 MB L2) over rotating input sets" %
                          (sum(4 * r.wl.N * r.esz * (r.nbuf if len(runners) == 1 else 1) for r in runners) >> 20),
-                   "timing": "median of %d regions of %d steps (%.2f s timed); CUDA events on the launch stream"
-                             % (len(regions), K, sum(regions) * 1e-3),
+                   "timing": "median of %d regions of %d steps (%.2f s timed), CUDA events on the launch stream around each "
+                             "region; per-call times from %d further regions with an event around every call (%.4f ms "
+                             "per step that way)" % (len(regions), K, sum(regions) * 1e-3, len(call_regions),
+                                                     statistics.median(call_regions) / K),
                    "parallelism": "dp%d (batch-sharded; one all-reduce of the flat parameter-gradient buffer per stage)" % world},
         "clocks": clocks,
         "ms_per_step_x_sm_mhz": ms_step * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,

@@ -163,14 +163,20 @@ wtconv_status wtconv_backward(const wtconv_desc *desc, const void *x, const void
 
 /* Device-side status of the last call that used `workspace` (device pointer; NULL = the array built into the
  * library that wtconv_backward_static uses, on the current device) with this descriptor: enqueues on
- * `stream` a copy of the workspace's status word into *h_flag (a HOST int32, pinned if the copy is to be
- * asynchronous).  Once the stream has reached this point, 0 means every bounded wait inside the kernels
- * completed (the paper's kernels wait for nothing; ours wait only for their own bulk copies); non-zero means a
- * wait ran out and the outputs of that call are not valid (report it as WTCONV_ERR_TIMEOUT).  For descriptors
- * served by the tiled kernels, which wait for nothing, *h_flag is set to 0 at once.  The library itself never
- * synchronises, so it cannot return that code from wtconv_forward / wtconv_backward.
+ * `stream` a one-thread kernel that evaluates the workspace's status words and a copy of the verdict into
+ * *h_flag (a HOST int32, pinned if the copy is to be asynchronous).  Once the stream has reached this point, 0
+ * means every bounded wait inside the kernels completed (the paper's kernels wait for nothing; ours wait only
+ * for their own bulk copies); non-zero means a wait ran out and the outputs of that call are not valid (report
+ * it as WTCONV_ERR_TIMEOUT).  For descriptors served by the tiled kernels, which wait for nothing, *h_flag is
+ * set to 0 at once.  The library itself never synchronises, so it cannot return that code from wtconv_forward /
+ * wtconv_backward.
+ * How the words work: no call clears them (a clearing operation between two kernels would keep the second from
+ * starting behind the tail of the first).  Every call stamps its launches with a fresh tag; a block whose wait
+ * ran out stores the tag in the first word, block 0 stores it in the second, and the two are equal only if the
+ * last call timed out.  A call replayed from a captured graph repeats its tag, so after one replay has timed out
+ * the later replays of that graph read as timed out as well.
  * Errors: NULL, the descriptor's own errors, ALIGNMENT (workspace), CUDA. */
-wtconv_status wtconv_read_status(const wtconv_desc *desc, const void *workspace, int32_t *h_flag, void *stream);
+wtconv_status wtconv_read_status(const wtconv_desc *desc, void *workspace, int32_t *h_flag, void *stream);
 
 /* Backward pass for callers that cannot hand over a workspace.  (The paper has no counterpart: it never
  * discusses where its kernels' scratch comes from.)
@@ -189,9 +195,10 @@ wtconv_status wtconv_read_status(const wtconv_desc *desc, const void *workspace,
  *     whole-plane kernels serve need well under 1 MiB, large planes on the tiled path need far more).
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
  *     device current); make that first call outside any stream capture.  Later calls on that device reuse it.
- *   - All calls on one device share the one array, and it keeps whatever the last call left in it.  Each call
- *     clears what has to start at zero, so stale contents are harmless, but two calls whose kernels overlap
- *     on the GPU (different streams) race on it: serialise them, or use wtconv_backward with two workspaces.
+ *   - All calls on one device share the one array, and it keeps whatever the last call left in it.  No call
+ *     depends on what it finds there (what must start at zero is cleared, the rest is written before it is
+ *     read), so stale contents are harmless, but two calls whose kernels overlap on the GPU (different
+ *     streams) race on it: serialise them, or use wtconv_backward with two workspaces.
  *   - The kernels' status word lives in the array too: read it with wtconv_read_status(desc, NULL, ...).
  *   - WTCONV_ERR_ARCH (device is not compute capability 10.x) is reported before the array is looked up. */
 #define WTCONV_STATIC_SCRATCH_BYTES (8u << 20)

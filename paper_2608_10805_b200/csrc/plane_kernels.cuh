@@ -129,6 +129,7 @@ struct Geom {
     int nthreads, nblocks, blocks_per_sm;
     int vec;                               // 1: W % 4 == 0, rows are staged with 4-element vector loads
     int no_copy;                           // test mode: bulk copies are never issued and waits give up quickly (the timeout path)
+    unsigned tag;                          // non-zero tag of the call this launch belongs to (status words, see common.cuh)
     int bulk;                              // 1: planes are fetched ahead with cp.async.bulk into a ring of raw buffers at raw_off
     int nstage, stage_bytes;               // ring depth (units in flight) and bytes per ring entry
     int raw_off, raw_slot_bytes, plane_bytes;  // raw staging buffer (float offset), bytes per plane slot / per plane
@@ -148,10 +149,7 @@ struct Geom {
 
 __host__ __device__ inline int pad4(int n) { return (n + 3) & ~3; }
 
-// Block containing unit v when `units` are split into `nb` contiguous ranges [iU/nb, (i+1)U/nb).
-__host__ __device__ inline int block_of_unit(long long v, int nb, int units) {
-    return (int)(((v + 1) * nb - 1) / units);
-}
+using wt::block_of_unit;
 
 // ------------------------------------------------------------------ shared device pieces
 __device__ __forceinline__ void build_weight_table(float *wtab, const Geom &g, int c0, bool flip,
@@ -590,7 +588,7 @@ __device__ __forceinline__ void start_prefetch(unsigned long long *bar, char *ra
 // copy lands in shared memory the block has already given back.
 __device__ __forceinline__ void give_up_after_timeout(unsigned long long *bar, const Geom &g, int ring, unsigned parity, int u,
                                                       int u_end, int *status) {
-    if (threadIdx.x == 0) atomicExch(status, 1);
+    if (threadIdx.x == 0) atomicExch(status + STATUS_TIMEOUT, (int)g.tag);
     const unsigned limit = g.no_copy ? WAIT_LIMIT_TEST : WAIT_LIMIT;
     for (int s = 0; s < g.nstage && u + s < u_end; ++s) {
         mbar_wait(bar + ring, parity, limit);
@@ -796,7 +794,6 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    if (g.bulk) start_prefetch<T>(bar, raw, g, x, nullptr, u_begin, u_end);
     zero_fill(sm, g);
     unsigned parity = 0;
     int ring = 0;  // ring entry the current unit arrives in
@@ -829,6 +826,12 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         items[k] = decode_item(g, hoist_items ? tid + k * nthr : 0x3fffffff, nlevel_items, nitems, bslot, tyy, txx, has_base);
     PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
     PatchD patch1 = decode_patch(g, g.offA, hoist_patch && srank < nstagers ? srank + nstagers : 0x3fffffff);
+    // Everything above touched shared memory and registers only and may have run beside the tail of the kernel
+    // before this one; global memory is used from here on.
+    dependents_may_start();
+    wait_for_predecessor();
+    if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
+    if (g.bulk) start_prefetch<T>(bar, raw, g, x, nullptr, u_begin, u_end);
     __syncthreads();
     // (channel group, image) of the current unit, carried along instead of divided out per unit
     int cg = u_begin / g.B, b = u_begin - cg * g.B;
@@ -953,7 +956,6 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    if (g.bulk) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
     zero_fill(sm, g);
     const int arrays_floats = g.raw_off;  // haloed arrays (and reduction scratch) end where the raw buffer starts
     unsigned parity = 0;
@@ -970,6 +972,10 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 #pragma unroll
     for (int t = 0; t < KK; ++t) acc[t] = 0.f;
     int ring = 0;
+    dependents_may_start();
+    wait_for_predecessor();  // shared memory and registers only up to here
+    if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
+    if (g.bulk) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
     __syncthreads();
     int c = u_begin / g.B, b = u_begin - c * g.B;  // this kernel is planned with one plane per unit: group = channel
     for (int u = u_begin; u < u_end; ++u, (++b == g.B ? (b = 0, ++c) : 0)) {
@@ -1102,7 +1108,6 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     char *raw = reinterpret_cast<char *>(sm + g.raw_off);
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
-    if (BULK) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
     zero_fill(sm, g);
     unsigned parity = 0;
     const int L = g.L, nlv = g.lvl_start[L + 1], ncls = 1 + 4 * L;
@@ -1130,6 +1135,10 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     for (int t = 0; t < KK; ++t) accw[t] = 0.f;
     int c_prev = -1;
     int ring = 0;
+    dependents_may_start();
+    wait_for_predecessor();  // shared memory and registers only up to here
+    if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
+    if (BULK) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
     __syncthreads();
     int cg = u_begin / g.B, b = u_begin - cg * g.B;
     for (int u = u_begin; u < u_end; ++u, (++b == g.B ? (b = 0, ++cg) : 0)) {
@@ -1715,8 +1724,8 @@ inline bool supported(int H, int W, int k, int L, int dtype) {
     return plan_forward(2, 2, H, W, L, dtype_bytes(dtype), g) && plan_wgrad(2, 2, H, W, L, dtype_bytes(dtype), g);
 }
 
-// Workspace: a status word (256 bytes reserved; nonzero after a run = a bounded wait on a copy barrier ran
-// out), then for backward the base partials [C][np][26] and the level partials [L][C][np][4][25] (float).
+// Workspace: the status words (256 bytes reserved; see common.cuh), then for backward the base partials
+// [C][np][26] and the level partials [L][C][np][4][25] (float).
 constexpr size_t STATUS_BYTES = 256;
 inline size_t forward_workspace_bytes(int, int, int, int, int) { return STATUS_BYTES; }
 inline size_t backward_workspace_bytes(int B, int C, int H, int W, int L, int elem_bytes, unsigned tune = 0) {
@@ -1749,7 +1758,9 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
     {                                                                                               \
         constexpr auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_, TH_>;                         \
         if ((e = opt_in_smem<kern>()) != cudaSuccess) return e;                                     \
-        kern<<<g.nblocks, g.nthreads, smem, st>>>(g, x, w0, s0, b0, wl, sl, out, status);           \
+        if ((e = launch_overlapped(kern, (unsigned)g.nblocks, (unsigned)g.nthreads, smem, st, g, x, w0, s0, b0, wl, sl, \
+                                   out, status)) != cudaSuccess)                                    \
+            return e;                                                                               \
     }
 #define WT_LAUNCH_FWD(MAXT_, MINB_) { if (g.th == 8) WT_LAUNCH_FWD_TH(MAXT_, MINB_, 8) else WT_LAUNCH_FWD_TH(MAXT_, MINB_, 4) }
     if (g.nthreads <= 128 && g.blocks_per_sm <= 3) {
@@ -1764,36 +1775,40 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
     return cudaGetLastError();
 }
 
+// `tag`: the call's status tag (non-zero, fresh per call).  Nothing is cleared and no other stream operation is
+// enqueued besides the kernel, so that the launch can overlap the tail of the kernel before it.
 template <typename T>
 cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
-                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tune = 0,
+                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tag, unsigned tune = 0,
                     bool no_copy = false) {
     Geom g;
     if (!plan_forward(B, C, H, W, L, (int)sizeof(T), g, tune)) return cudaErrorInvalidValue;
     g.no_copy = no_copy;
-    cudaError_t e = cudaMemsetAsync(ws, 0, STATUS_BYTES, st);
-    if (e != cudaSuccess) return e;
+    g.tag = tag;
     return launch_fwd<T, false>(g, x, w0, s0, b0, wl, sl, out, reinterpret_cast<int *>(ws), st);
 }
 
+// The epilogue learns from `ep` which partial slots the blocks wrote (EpiloguePtrs::grp), so nothing is cleared here
+// either.
 template <typename T>
 cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go, const float *w0, const float *s0,
-                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st,
+                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st, unsigned tag,
                      unsigned tune = 0, bool no_copy = false) {
     Geom gw, gf;
+    cudaError_t e;
     if (plan_bwd_fused(B, C, H, W, L, (int)sizeof(T), gw, tune)) {
         gw.no_copy = no_copy;
+        gw.tag = tag;
         float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
         float *partl = part0 + (size_t)C * gw.np * (KK + 1);
-        const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
-        cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // partial slots no block writes must read as zero
-        if (e != cudaSuccess) return e;
 #define WT_LAUNCH_BWD(TH_, BULK_)                                                                          \
     {                                                                                                      \
         constexpr auto kb = plane_bwd_kernel<T, TH_, BULK_>;                                               \
         if ((e = opt_in_smem<kb>()) != cudaSuccess) return e;                                              \
-        kb<<<gw.nblocks, gw.nthreads, (size_t)gw.smem_floats * 4, st>>>(gw, x, go, w0, s0, wl, sl, gx, part0, partl, \
-                                                                         reinterpret_cast<int *>(ws));     \
+        if ((e = launch_overlapped(kb, (unsigned)gw.nblocks, (unsigned)gw.nthreads, (size_t)gw.smem_floats * 4, st, gw, \
+                                   x, go, w0, s0, wl, sl, gx, part0, partl, reinterpret_cast<int *>(ws))) !=  \
+            cudaSuccess)                                                                                   \
+            return e;                                                                                      \
     }
         if (gw.th == 8) {
             if (gw.bulk == 2) WT_LAUNCH_BWD(8, 2) else WT_LAUNCH_BWD(8, 0)
@@ -1808,23 +1823,24 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
             ep->partl[l] = partl + (size_t)l * C * gw.np * 4 * KK;
             ep->npl[l] = gw.np;
         }
+        ep->grp = gw.NPL; ep->B = B; ep->units = gw.units; ep->nblocks = gw.nblocks;
         return cudaSuccess;
     }
     if (!plan_wgrad(B, C, H, W, L, (int)sizeof(T), gw, tune) || !plan_forward(B, C, H, W, L, (int)sizeof(T), gf, tune))
         return cudaErrorInvalidValue;
     gw.no_copy = gf.no_copy = no_copy;
+    gw.tag = gf.tag = tag;
     int *status = reinterpret_cast<int *>(ws);
     float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
     float *partl = part0 + (size_t)C * gw.np * (KK + 1);
-    const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), tune);
-    cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // status word; partial slots no block writes must read as zero
-    if (e != cudaSuccess) return e;
     const size_t smem = (size_t)gw.smem_floats * 4;
 #define WT_LAUNCH_WG(MAXT_, MINB_, TH_)                                                            \
     {                                                                                              \
         constexpr auto kw = plane_wgrad_kernel<T, MAXT_, MINB_, TH_>;                              \
         if ((e = opt_in_smem<kw>()) != cudaSuccess) return e;                                      \
-        kw<<<gw.nblocks, gw.nthreads, smem, st>>>(gw, x, go, part0, partl, status);                \
+        if ((e = launch_overlapped(kw, (unsigned)gw.nblocks, (unsigned)gw.nthreads, smem, st, gw, x, go, part0, partl, \
+                                   status)) != cudaSuccess)                                        \
+            return e;                                                                              \
     }
     if (gw.nthreads <= 128) {
         if (gw.th == 8) WT_LAUNCH_WG(128, 4, 8) else WT_LAUNCH_WG(128, 4, 4)
@@ -1840,6 +1856,7 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         ep->partl[l] = partl + (size_t)l * C * gw.np * 4 * KK;
         ep->npl[l] = gw.np;
     }
+    ep->grp = gw.NPL; ep->B = B; ep->units = gw.units; ep->nblocks = gw.nblocks;
     return cudaSuccess;
 }
 
@@ -1847,10 +1864,11 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
 // activation type: the kernels are compiled once, in the instantiation unit of that type.
 #define WT_PLANE_INSTANTIATE(T, EXTERN)                                                                                    \
     EXTERN template cudaError_t forward<T>(int, int, int, int, int, const T *, const float *, const float *, const float *, \
-                                           const float *, const float *, T *, char *, cudaStream_t, unsigned, bool);       \
+                                           const float *, const float *, T *, char *, cudaStream_t, unsigned, unsigned,    \
+                                           bool);                                                                          \
     EXTERN template cudaError_t backward<T>(int, int, int, int, int, const T *, const T *, const float *, const float *,    \
                                             const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t,       \
-                                            unsigned, bool);
+                                            unsigned, unsigned, bool);
 
 }  // namespace plane
 }  // namespace wt

@@ -63,6 +63,7 @@ struct TGeom {
     int nteams, nthreads, nblocks, units, ngroups, np;
     int th;
     int no_copy;
+    unsigned tag;                           // non-zero tag of the call this launch belongs to (status words)
     double score;
 };
 
@@ -298,6 +299,11 @@ team_kernel(const __grid_constant__ TGeom g, const T *__restrict__ x, const T *_
         plane::fence_async_smem();  // the zero fill (generic proxy) is ordered before the first bulk copies into the ring
     }
     __syncthreads();
+    // The set-up above touched shared memory and registers only and may have run beside the tail of the kernel
+    // before this one; global memory is used from here on.
+    dependents_may_start();
+    wait_for_predecessor();
+    if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
 
     const int u_begin = (int)((long long)blockIdx.x * g.units / gridDim.x);
     const int u_end = (int)((long long)(blockIdx.x + 1) * g.units / gridDim.x);
@@ -374,7 +380,7 @@ team_kernel(const __grid_constant__ TGeom g, const T *__restrict__ x, const T *_
             }
             if (team_sync_or(tw, bar_id, late)) {  // a copy never landed: record it and stop working (see the end of the kernel)
                 dead = true;
-                if (lt == 0) atomicExch(status, 1);
+                if (lt == 0) atomicExch(status + STATUS_TIMEOUT, (int)g.tag);
                 break;
             }
             if (lt == 0 && u + NSTAGE * nteams < seg_end) {  // the ring entry is free again: fetch the unit two rounds ahead
@@ -690,38 +696,39 @@ cudaError_t launch(const TGeom &g, const T *x, const T *go, const float *w0, con
     if (g.th == 7) {
         constexpr auto kern = team_kernel<T, 7, BWD>;
         if ((e = plane::opt_in_smem<kern>()) != cudaSuccess) return e;
-        kern<<<g.nblocks, g.nthreads, g.smem_bytes, st>>>(g, x, go, w0, s0, b0, wl, sl, out, part0, partl, status);
+        e = launch_overlapped(kern, (unsigned)g.nblocks, (unsigned)g.nthreads, (size_t)g.smem_bytes, st, g, x, go, w0, s0, b0, wl,
+                              sl, out, part0, partl, status);
     } else {
         constexpr auto kern = team_kernel<T, 4, BWD>;
         if ((e = plane::opt_in_smem<kern>()) != cudaSuccess) return e;
-        kern<<<g.nblocks, g.nthreads, g.smem_bytes, st>>>(g, x, go, w0, s0, b0, wl, sl, out, part0, partl, status);
+        e = launch_overlapped(kern, (unsigned)g.nblocks, (unsigned)g.nthreads, (size_t)g.smem_bytes, st, g, x, go, w0, s0, b0, wl,
+                              sl, out, part0, partl, status);
     }
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <typename T>
 cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
-                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, bool no_copy, int forceG) {
+                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tag, bool no_copy,
+                    int forceG) {
     TGeom g;
     if (!plan(B, C, H, W, L, (int)sizeof(T), false, g, forceG)) return cudaErrorInvalidValue;
     g.no_copy = no_copy;
-    cudaError_t e = cudaMemsetAsync(ws, 0, plane::STATUS_BYTES, st);
-    if (e != cudaSuccess) return e;
+    g.tag = tag;  // nothing is cleared: see the status words in common.cuh
     return launch<T, false>(g, x, nullptr, w0, s0, b0, wl, sl, out, nullptr, nullptr, reinterpret_cast<int *>(ws), st);
 }
 
 template <typename T>
 cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go, const float *w0, const float *s0,
-                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st, bool no_copy,
-                     int forceG) {
+                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st, unsigned tag,
+                     bool no_copy, int forceG) {
     TGeom g;
     if (!plan(B, C, H, W, L, (int)sizeof(T), true, g, forceG)) return cudaErrorInvalidValue;
     g.no_copy = no_copy;
+    g.tag = tag;
     float *part0 = reinterpret_cast<float *>(ws + plane::STATUS_BYTES);
     float *partl = part0 + (size_t)C * g.np * (KK + 1);
-    const size_t pbytes = backward_workspace_bytes(B, C, H, W, L, (int)sizeof(T), forceG);
-    cudaError_t e = cudaMemsetAsync(ws, 0, pbytes, st);  // status word; partial slots no block writes must read as zero
-    if (e != cudaSuccess) return e;
+    cudaError_t e;  // nothing is cleared: the epilogue is told which partial slots the blocks write
     if ((e = launch<T, true>(g, x, go, w0, s0, nullptr, wl, sl, gx, part0, partl, reinterpret_cast<int *>(ws), st)) != cudaSuccess)
         return e;
     ep->part0 = part0;
@@ -730,15 +737,16 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         ep->partl[l] = partl + (size_t)l * C * g.np * 4 * KK;
         ep->npl[l] = g.np;
     }
+    ep->grp = g.G; ep->B = B; ep->units = g.units; ep->nblocks = g.nblocks;
     return cudaSuccess;
 }
 
 #define WT_TEAM_INSTANTIATE(T, EXTERN)                                                                                     \
     EXTERN template cudaError_t forward<T>(int, int, int, int, int, const T *, const float *, const float *, const float *, \
-                                           const float *, const float *, T *, char *, cudaStream_t, bool, int);            \
+                                           const float *, const float *, T *, char *, cudaStream_t, unsigned, bool, int);  \
     EXTERN template cudaError_t backward<T>(int, int, int, int, int, const T *, const T *, const float *, const float *,    \
-                                            const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t, bool, \
-                                            int);
+                                            const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t,       \
+                                            unsigned, bool, int);
 
 }  // namespace team
 }  // namespace wt

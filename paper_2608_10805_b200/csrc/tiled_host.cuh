@@ -127,6 +127,7 @@ inline wtconv_status launch_epilogue(const wtconv_desc *d, const wt::EpiloguePtr
                               float *gwl, float *gsl, cudaStream_t st) {
     const int KK = d->k * d->k;
     size_t smem = sizeof(double) * (KK + 1 + (size_t)d->L * 4 * KK);
+    // an ordinary launch: it starts when the kernels that produced the partial sums have completed
     wt::unfold_epilogue_kernel<0><<<d->C, 128, smem, st>>>(d->C, d->k, d->L, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl,
                                                         gsl);
     return launch_status();

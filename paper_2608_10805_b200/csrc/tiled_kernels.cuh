@@ -812,6 +812,11 @@ struct EpiloguePtrs {
     int np0;
     const float *partl[8];
     int npl[8];
+    // Which of a channel's slots hold sums.  grp == 0: all of them (the producer cleared the rest).  grp > 0: the
+    // producer was a persistent kernel whose `nblocks` blocks split `units` = (C / grp) x B work units (grp channels
+    // of one image each, channel-group major) into contiguous ranges; slot i of a channel belongs to the i-th block
+    // whose range meets the channel's group, later slots were never written and are not read.
+    int grp, B, units, nblocks;
 };
 
 template <int UNUSED>  // a template only so that every translation unit may include this header
@@ -823,15 +828,23 @@ unfold_epilogue_kernel(int C, int K, int L, EpiloguePtrs ep, const float *__rest
     extern __shared__ double folded[];  // [KK+1] base, then [L][4][KK]
     const int c = blockIdx.x, KK = K * K;
     const int n0 = KK + 1, nl = 4 * KK;
+    dependents_may_start();  // the next kernel on the stream may run its set-up beside this one
+    int written = 0x7fffffff;  // slots of this channel that hold sums
+    if (ep.grp > 0) {
+        const long long first_unit = (long long)(c / ep.grp) * ep.B;
+        written = block_of_unit(first_unit + ep.B - 1, ep.nblocks, ep.units) - block_of_unit(first_unit, ep.nblocks, ep.units) + 1;
+    }
     for (int e = threadIdx.x; e < n0 + L * nl; e += blockDim.x) {
         double acc = 0.0;
         if (e < n0) {
             const float *q = ep.part0 + (size_t)c * ep.np0 * n0 + e;
-            for (int i = 0; i < ep.np0; ++i) acc += (double)q[(size_t)i * n0];
+            const int n = ep.np0 < written ? ep.np0 : written;
+            for (int i = 0; i < n; ++i) acc += (double)q[(size_t)i * n0];
         } else {
             int l = (e - n0) / nl, t = (e - n0) - l * nl;
             const float *q = ep.partl[l] + (size_t)c * ep.npl[l] * nl + t;
-            for (int i = 0; i < ep.npl[l]; ++i) acc += (double)q[(size_t)i * nl];
+            const int n = ep.npl[l] < written ? ep.npl[l] : written;
+            for (int i = 0; i < n; ++i) acc += (double)q[(size_t)i * nl];
         }
         folded[e] = acc;
     }

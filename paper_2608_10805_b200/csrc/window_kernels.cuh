@@ -553,7 +553,7 @@ cudaError_t launch_window(const WGeom &w, const T *x, const T *go, const float *
 
 template <typename T>
 cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
-                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st) {
+                    const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tag) {
     WGeom w;
     if (!make_plan(B, C, H, W, L, (int)sizeof(T), false, w)) return cudaErrorInvalidValue;
     const WsPlan p = ws_plan(B, C, H, W, L, (int)sizeof(T));
@@ -568,7 +568,7 @@ cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *
         fill_f32_kernel<<<(C + 255) / 256, 256, 0, st>>>(ones, 1.f, (size_t)C);
         // levels 3..L of x are levels 1..L-2 of the carrier; its base path is switched off by zero weights
         if ((e = plane::forward<float>(B, C, w.H2, w.W2, L - 2, X2, zeros, ones, nullptr, wl + (size_t)2 * C * 4 * KK, sl + (size_t)2 * C * 4,
-                                       R3, ws + p.deep, st, 0, false)) != cudaSuccess)
+                                       R3, ws + p.deep, st, tag, 0, false)) != cudaSuccess)
             return e;
         add = R3;
     }
@@ -577,7 +577,7 @@ cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *
 
 template <typename T>
 cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go, const float *w0, const float *s0,
-                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st) {
+                     const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st, unsigned tag) {
     WGeom w;
     if (!make_plan(B, C, H, W, L, (int)sizeof(T), true, w)) return cudaErrorInvalidValue;
     const WsPlan p = ws_plan(B, C, H, W, L, (int)sizeof(T));
@@ -596,8 +596,10 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         fill_f32_kernel<<<(C + 255) / 256, 256, 0, st>>>(ones, 1.f, (size_t)C);
         EpiloguePtrs deep = {};
         char *deep_ws = ws + p.deep;
+        // the epilogue reads every slot of the merged partial sums: the slots the carrier's kernels do not write are zero
+        if ((e = cudaMemsetAsync(deep_ws, 0, plane::backward_workspace_bytes(B, C, w.H2, w.W2, L - 2, 4), st)) != cudaSuccess) return e;
         if ((e = plane::backward<float>(B, C, w.H2, w.W2, L - 2, X2, G2, zeros, ones, wl + (size_t)2 * C * 4 * KK, sl + (size_t)2 * C * 4, gX2,
-                                        deep_ws, &deep, st, 0, false)) != cudaSuccess)
+                                        deep_ws, &deep, st, tag, 0, false)) != cudaSuccess)
             return e;
         for (int l = 2; l < L; ++l) { ep->partl[l] = deep.partl[l - 2]; ep->npl[l] = deep.npl[l - 2]; }
         add = gX2;
@@ -611,9 +613,10 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
 
 #define WT_WINDOW_INSTANTIATE(T, EXTERN)                                                                                   \
     EXTERN template cudaError_t forward<T>(int, int, int, int, int, const T *, const float *, const float *, const float *, \
-                                           const float *, const float *, T *, char *, cudaStream_t);                       \
+                                           const float *, const float *, T *, char *, cudaStream_t, unsigned);             \
     EXTERN template cudaError_t backward<T>(int, int, int, int, int, const T *, const T *, const float *, const float *,    \
-                                            const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t);
+                                            const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t,       \
+                                            unsigned);
 
 }  // namespace window
 }  // namespace wt

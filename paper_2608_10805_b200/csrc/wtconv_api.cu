@@ -11,6 +11,8 @@
 #include "tiled_host.cuh"
 #include "reference_chain.cuh"
 
+#include <atomic>
+#include <chrono>
 #include <mutex>
 
 namespace wt {
@@ -80,6 +82,24 @@ wtconv_status check_device() {
     return major == 10 ? WTCONV_OK : WTCONV_ERR_ARCH;
 }
 
+// ------------------------------------------------------------------ status tags
+// Every call that launches kernels with bounded waits carries a fresh non-zero tag (see the status words in
+// common.cuh).  The sequence starts at a clock-derived value, so that tags left in a workspace by another process or
+// an earlier load of the library are unlikely to repeat.
+unsigned next_status_tag() {
+    static std::atomic<unsigned> counter{
+        (unsigned)std::chrono::steady_clock::now().time_since_epoch().count() * 2654435761u};
+    unsigned t = counter.fetch_add(1u, std::memory_order_relaxed) + 1u;
+    if (t == 0u) t = counter.fetch_add(1u, std::memory_order_relaxed) + 1u;
+    return t;
+}
+
+// 1 if the last call on this workspace recorded a timeout, else 0, into the third status word.
+__global__ void resolve_status_kernel(int *status) {
+    const int timeout = status[wt::STATUS_TIMEOUT], launch = status[wt::STATUS_LAUNCH];
+    status[wt::STATUS_RESOLVED] = (launch != 0 && timeout == launch) ? 1 : 0;
+}
+
 // ------------------------------------------------------------------ dispatch
 int team_force_g(const wtconv_desc *d) { return (int)((d->flags >> 16) & 63u); }  // "planes per work unit" override
 bool use_ref_chain(const wtconv_desc *d) { return (d->flags & WTCONV_FLAG_REFERENCE_CHAIN) != 0; }
@@ -111,20 +131,23 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
     if constexpr (K == 5) {
         if (use_team_path(d))
             return wt::team::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st,
-                                        (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, team_force_g(d)) == cudaSuccess
+                                        next_status_tag(), (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0,
+                                        team_force_g(d)) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
     if constexpr (K == 5) {
         if (use_window_path(d))
-            return wt::window::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st) == cudaSuccess
+            return wt::window::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st,
+                                          next_status_tag()) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
     if (use_plane_path(d)) {
         if constexpr (K == 5)
             return wt::plane::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws,
-                                         st, d->flags >> 8, (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) == cudaSuccess
+                                         st, next_status_tag(), d->flags >> 8,
+                                         (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
@@ -142,7 +165,8 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
         if (use_team_path(d)) {
             wt::EpiloguePtrs ep = {};
             if (wt::team::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl, (T *)gx,
-                                      ws, &ep, st, (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, team_force_g(d)) != cudaSuccess)
+                                      ws, &ep, st, next_status_tag(), (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0,
+                                      team_force_g(d)) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
         }
@@ -151,7 +175,7 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
         if (use_window_path(d)) {
             wt::EpiloguePtrs ep = {};
             if (wt::window::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl, (T *)gx, ws, &ep,
-                                        st) != cudaSuccess)
+                                        st, next_status_tag()) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
         }
@@ -160,7 +184,7 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
         if constexpr (K == 5) {
             wt::EpiloguePtrs ep = {};
             if (wt::plane::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl,
-                                       (T *)gx, ws, &ep, st, d->flags >> 8,
+                                       (T *)gx, ws, &ep, st, next_status_tag(), d->flags >> 8,
                                        (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
@@ -588,7 +612,7 @@ wtconv_status wtconv_step_host(const wtconv_desc *d, const void *h_x, const void
     return ok ? WTCONV_OK : WTCONV_ERR_CUDA;
 }
 
-wtconv_status wtconv_read_status(const wtconv_desc *d, const void *workspace, int32_t *h_flag, void *stream) {
+wtconv_status wtconv_read_status(const wtconv_desc *d, void *workspace, int32_t *h_flag, void *stream) {
     wtconv_status st = validate_desc(d);
     if (st != WTCONV_OK) return st;
     if (!h_flag) return WTCONV_ERR_NULL;
@@ -600,13 +624,18 @@ wtconv_status wtconv_read_status(const wtconv_desc *d, const void *workspace, in
     }
     if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
     if (use_window_path(d) && d->L > 2)  // the carrier's whole-plane kernels keep the only status word of this path
-        workspace = (const char *)workspace + wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).deep;
+        workspace = (char *)workspace + wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).deep;
     else if (!use_plane_path(d)) {  // the tiled, window (L <= 2) and reference kernels wait for nothing and keep no status word
         *h_flag = 0;
         return WTCONV_OK;
     }
-    // the status word is the first word of every workspace the plane kernels use
-    return cudaMemcpyAsync(h_flag, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream) == cudaSuccess
+    // the status words open every workspace the plane kernels use: compare the timeout tag with the tag of the
+    // last launch on the device, then fetch the verdict
+    int *words = (int *)workspace;
+    resolve_status_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(words);
+    if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
+    return cudaMemcpyAsync(h_flag, words + wt::STATUS_RESOLVED, sizeof(int32_t), cudaMemcpyDeviceToHost,
+                           (cudaStream_t)stream) == cudaSuccess
                ? WTCONV_OK
                : WTCONV_ERR_CUDA;
 }
@@ -621,8 +650,8 @@ wtconv_status wtconv_backward_static(const wtconv_desc *d, const void *x, const 
     if ((st = check_device()) != WTCONV_OK) return st;
     void *scratch = nullptr;
     if ((st = static_scratch_for_current_device(&scratch)) != WTCONV_OK) return st;
-    // wtconv_backward clears the parts of its workspace that must start at zero on every call, so the
-    // contents a previous call left in the shared array do not matter.
+    // wtconv_backward never depends on what it finds in its workspace, so the contents a previous call left in
+    // the shared array do not matter.
     return wtconv_backward(d, x, grad_out, w0, s0, b0, wl, sl, grad_x, grad_w0, grad_s0, grad_b0, grad_wl, grad_sl,
                            scratch, (size_t)WTCONV_STATIC_SCRATCH_BYTES, stream);
 }
