@@ -202,48 +202,49 @@ class Runner:
                 "training_step_peak": 4 * act + 2 * par + max(self.ws_fwd, self.ws_bwd)}
 
 
-def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions, direction="both",
-                 per_call=True):
-    """Regions of exactly K steps, repeated until `min_seconds` have been timed.  per_call: every library call is
-    bracketed by events as well (an event between two kernels keeps the second from starting behind the tail of the
-    first, so regions timed this way run a little longer than a plain sequence of calls).
-    Returns (region_ms list, per-runner [fwd_ms list, bwd_ms list])."""
-    def step(i, ev=None):
-        for j, r in enumerate(runners):
-            if ev is not None:
-                ev[j][0].record(stream)
+def time_regions(runners, K, warmup, stream, torch, sync_all, all_reduce, min_seconds, max_regions, direction="both"):
+    """Milliseconds of regions of exactly K steps (nothing but the library calls and the gradient exchange on the
+    stream), repeated until `min_seconds` have been timed."""
+    def step(i):
+        for r in runners:
             if direction != "bwd":
                 r.fwd(i, stream)
-            if ev is not None:
-                ev[j][1].record(stream)
             if direction != "fwd":
                 r.bwd(i, stream)
-            if ev is not None:
-                ev[j][2].record(stream)
             all_reduce(r)
     for i in range(warmup):
         step(i)
     sync_all()
-    regions, fwd, bwd = [], [[] for _ in runners], [[] for _ in runners]
-    total = 0.0
+    regions, total = [], 0.0
     while len(regions) < max_regions and (total < min_seconds or not regions):
-        evs = [[tuple(torch.cuda.Event(enable_timing=True) for _ in range(3)) for _ in runners] if per_call else None
-               for _ in range(K)]
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         sync_all()
         e0.record(stream)
         for i in range(K):
-            step(i, evs[i])
+            step(i)
         e1.record(stream)
         sync_all()
-        ms = e0.elapsed_time(e1)
-        regions.append(ms)
-        total += ms * 1e-3
-        for ev in evs if per_call else []:
-            for j in range(len(runners)):
-                fwd[j].append(ev[j][0].elapsed_time(ev[j][1]))
-                bwd[j].append(ev[j][1].elapsed_time(ev[j][2]))
-    return regions, fwd, bwd
+        regions.append(e0.elapsed_time(e1))
+        total += regions[-1] * 1e-3
+    return regions
+
+
+def time_calls(fn, K, reps, stream, torch, sync_all):
+    """Milliseconds per call: median over `reps` regions of K consecutive calls of one kind with nothing between them
+    on the stream (as in a training loop, a call may start its set-up behind the tail of the call before it)."""
+    for i in range(2):
+        fn(i)
+    sync_all()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(K):
+            fn(i)
+        e1.record(stream)
+        sync_all()
+        ts.append(e0.elapsed_time(e1) / K)
+    return statistics.median(ts)
 
 
 def row_for(r, fwd_ms, bwd_ms, peaks, io_model):
@@ -282,18 +283,8 @@ PAPER_FWD_RATIO_F32 = [3.67, 4.20, 4.32, 4.35, 4.37]
 def comparator_rows(names, mk, wt, io_model, stream, torch, sync_all, have):
     """Reference-style chain and ablation steps next to the fused kernels, one row per workload."""
     REF, FA, CS = wt.FLAG_REFERENCE_CHAIN, wt.FLAG_ABLATE_FUSED_ANALYSIS, wt.FLAG_ABLATE_COLLAPSED_SYNTHESIS
-    med = statistics.median
-
-    def timed(fn, reps):
-        for i in range(2):
-            fn(i)
-        sync_all()
-        ts = []
-        for i in range(reps):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream); fn(i); e1.record(stream); sync_all()
-            ts.append(e0.elapsed_time(e1) * 1e3)
-        return med(ts)
+    def timed(fn, reps):  # the protocol of the fused rows: consecutive calls, nothing between them
+        return time_calls(fn, 3, reps, stream, torch, sync_all) * 1e3
 
     out = []
     for name in names:
@@ -404,14 +395,13 @@ def main():
         time.sleep(0.2)
     t0 = time.time()
     # the headline: plain sequences of calls, nothing between them on the stream
-    regions, _, _ = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400, args.direction,
-                                 per_call=False)
-    # the per-call split behind the roofline entries: the same steps with an event around every call
-    call_regions, fwd_ms, bwd_ms = time_regions(runners, K, 0, stream, torch, sync_all, all_reduce, 0.1 if args.min_seconds else 0.0,
-                                                50, args.direction)
-    if args.direction != "both":  # a profiling run: the untimed call would divide by zero in the roofline rows
-        fwd_ms = [[max(v, 1e-6) for v in f] for f in fwd_ms]
-        bwd_ms = [[max(v, 1e-6) for v in b] for b in bwd_ms]
+    regions = time_regions(runners, K, W, stream, torch, sync_all, all_reduce, args.min_seconds, 400, args.direction)
+    # the per-call split behind the roofline entries: each call of the step on its own, K in a row
+    if args.direction == "both":
+        fwd_ms = [time_calls(lambda i, r=r: r.fwd(i, stream), K, 5, stream, torch, sync_all) for r in runners]
+        bwd_ms = [time_calls(lambda i, r=r: r.bwd(i, stream), K, 5, stream, torch, sync_all) for r in runners]
+    else:  # a profiling run of one direction: no split
+        fwd_ms = bwd_ms = [1e-6 for _ in runners]
     t1 = time.time()
     med = statistics.median(regions)
     ms = torch.tensor([med], device=dev)
@@ -466,8 +456,7 @@ def main():
     ms_step = ms_region / K
     n_step = sum(r.wl.N for r in runners)
     value = n_step * world / (ms_step * 1e-3)
-    mean = lambda v: sum(v) / len(v)
-    rows = [row_for(r, statistics.median(f), statistics.median(b), peaks, io_model) for r, f, b in zip(runners, fwd_ms, bwd_ms)]
+    rows = [row_for(r, f, b, peaks, io_model) for r, f, b in zip(runners, fwd_ms, bwd_ms)]
     fl_step = sum(io_model.algorithmic_flops(r.wl.B, r.wl.C, r.wl.H, r.wl.W, r.wl.k, r.wl.L, "fwd+bwd") for r in runners)
     by_step = sum(io_model.compulsory_bytes(r.wl.N, r.esz, "fwd+bwd") for r in runners)
     alu_floor_ms = fl_step / (FP32_ALU_PEAK_TFLOPS * 1e12) * 1e3
@@ -477,13 +466,13 @@ def main():
     def call_entry(j, kind):
         r_, row_ = runners[j], rows[j]
         f_ = io_model.algorithmic_flops(r_.wl.B, r_.wl.C, r_.wl.H, r_.wl.W, r_.wl.k, r_.wl.L, "fwd")
-        ms_, fl_ = (mean(bwd_ms[j]), 2 * f_) if kind == "backward" else (mean(fwd_ms[j]), f_)
+        ms_, fl_ = (bwd_ms[j], 2 * f_) if kind == "backward" else (fwd_ms[j], f_)
         ach_ = fl_ / (ms_ * 1e-3) / 1e12
         return {"bound": row_["bound"], "kernel": "%s call of %s (%s kernels)" % (kind, r_.wl.name, r_.plan),
                 "achieved": ach_, "peak": FP32_ALU_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": ach_ / FP32_ALU_PEAK_TFLOPS,
                 "traffic": NCU_DRAM_TRAFFIC.get((r_.wl.name, "plane_bwd" if kind == "backward" else "plane_fwd")),
                 "peak_source": PEAK_SOURCE, "launch_ms": ms_, "flops_per_launch": fl_,
-                "share_of_step": ms_ / (sum(mean(v) for v in fwd_ms) + sum(mean(v) for v in bwd_ms))}
+                "share_of_step": ms_ / (sum(fwd_ms) + sum(bwd_ms))}
     calls = [call_entry(j, kind) for j in range(len(rows)) for kind in ("forward", "backward")]
     dominant = max(calls, key=lambda c_: c_["launch_ms"])
     worst_call = min(calls, key=lambda c_: c_["frac"])
@@ -497,9 +486,9 @@ def main():
                    "l2": "a step touches %d MB (> 126 MB L2) over rotating input sets" %
                          (sum(4 * r.wl.N * r.esz * (r.nbuf if len(runners) == 1 else 1) for r in runners) >> 20),
                    "timing": "median of %d regions of %d steps (%.2f s timed), CUDA events on the launch stream around each "
-                             "region; per-call times from %d further regions with an event around every call (%.4f ms "
-                             "per step that way)" % (len(regions), K, sum(regions) * 1e-3, len(call_regions),
-                                                     statistics.median(call_regions) / K),
+                             "region, nothing between the calls; per-call times: median of 5 regions of %d consecutive "
+                             "calls of that kind (their sum: %.4f ms per step)"
+                             % (len(regions), K, sum(regions) * 1e-3, K, sum(fwd_ms) + sum(bwd_ms)),
                    "parallelism": "dp%d (batch-sharded; one all-reduce of the flat parameter-gradient buffer per stage)" % world},
         "clocks": clocks,
         "ms_per_step_x_sm_mhz": ms_step * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,
@@ -539,8 +528,9 @@ def main():
                 continue
             r = mk(inputs.WORKLOADS[name])
             k = 3 if r.wl.N > (1 << 27) else 10
-            _, f, b = time_regions([r], k, 3, stream, torch, sync_all, lambda _r: None, 0.05, 20)
-            table.append(row_for(r, statistics.median(f[0]), statistics.median(b[0]), peaks, io_model))
+            f = time_calls(lambda i: r.fwd(i, stream), k, 5, stream, torch, sync_all)
+            b = time_calls(lambda i: r.bwd(i, stream), k, 5, stream, torch, sync_all)
+            table.append(row_for(r, f, b, peaks, io_model))
             del r
             torch.cuda.empty_cache()
         result["per_workload"] = table

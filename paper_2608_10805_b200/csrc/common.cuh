@@ -50,9 +50,11 @@ __host__ __device__ inline int block_of_unit(long long v, int nb, int units) {
 // predecessor gave back, run their set-up (shared memory and registers only), and stop at
 // wait_for_predecessor(), which returns once the predecessor has completed and its writes are visible.  Every
 // access to global memory comes after that call.  dependents_may_start() lets the next kernel on the stream do the
-// same with respect to this one; both are no-ops in a kernel that was launched the ordinary way.  Only the persistent
-// kernels are launched this way: measured on B200, starting the small parameter-gradient epilogue early as well made
-// the training step of the four-stage set 4 % slower, while the persistent kernels alone gained 2 %.
+// same with respect to this one; both are no-ops in a kernel that was launched the ordinary way.  When to release the
+// dependents matters: a persistent kernel's blocks must all become resident together (each owns a fixed share of the
+// work), so nothing small may be let in early that would occupy part of an SM when they arrive.  Measured on B200 over
+// the four-stage training step: forward kernels releasing at their start and backward kernels (followed by the small
+// parameter-gradient epilogue) at their end gained 3 %; releasing the epilogue early cost 4 %.
 __device__ __forceinline__ void dependents_may_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

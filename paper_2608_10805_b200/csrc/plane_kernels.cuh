@@ -827,8 +827,9 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
     PatchD patch1 = decode_patch(g, g.offA, hoist_patch && srank < nstagers ? srank + nstagers : 0x3fffffff);
     // Everything above touched shared memory and registers only and may have run beside the tail of the kernel
-    // before this one; global memory is used from here on.
-    dependents_may_start();
+    // before this one; global memory is used from here on.  The input-gradient instantiation is followed by the small
+    // epilogue and releases it at the end (see plane_bwd_kernel).
+    if (!FLIP) dependents_may_start();
     wait_for_predecessor();
     if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
     if (g.bulk) start_prefetch<T>(bar, raw, g, x, nullptr, u_begin, u_end);
@@ -938,6 +939,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         // The next unit's staging overwrites x / Y (last read before the barrier above) and possibly the
         // weight table (bias already in a register); Z is next written after the staging barriers.
     }
+    if (FLIP) dependents_may_start();
     if (g.bulk_out && tid == 0) bulk_store_wait_read();  // shared memory must outlive the last bulk store's reads
 }
 
@@ -1135,8 +1137,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     for (int t = 0; t < KK; ++t) accw[t] = 0.f;
     int c_prev = -1;
     int ring = 0;
-    dependents_may_start();
-    wait_for_predecessor();  // shared memory and registers only up to here
+    wait_for_predecessor();  // shared memory and registers only up to here (dependents are released at the end)
     if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
     if (BULK) start_prefetch<T>(bar, raw, g, x, go, u_begin, u_end);
     __syncthreads();
@@ -1313,6 +1314,9 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
         // follows the tile phase) while the base-tile threads may still run this unit's synthesis, which
         // reads only Z (next written after the staging barriers) and registers.
     }
+    // The kernel behind this one is the small parameter-gradient epilogue: released any earlier, its blocks would sit
+    // on the SMs whose blocks finish first and keep the next persistent kernel from spreading over all SMs at once.
+    dependents_may_start();
     if (BULK && g.bulk_out && tid == 0) bulk_store_wait_read();
 }
 

@@ -301,7 +301,7 @@ team_kernel(const __grid_constant__ TGeom g, const T *__restrict__ x, const T *_
     __syncthreads();
     // The set-up above touched shared memory and registers only and may have run beside the tail of the kernel
     // before this one; global memory is used from here on.
-    dependents_may_start();
+    if (!BWD) dependents_may_start();  // backward: at the end (the kernel behind it is the small epilogue, see plane_bwd_kernel)
     wait_for_predecessor();
     if (blockIdx.x == 0 && tid == 0) status[STATUS_LAUNCH] = (int)g.tag;
 
@@ -521,6 +521,7 @@ team_kernel(const __grid_constant__ TGeom g, const T *__restrict__ x, const T *_
         }
         seg = seg_end;
     }
+    if (BWD) dependents_may_start();
     if (lt == 0) plane::bulk_store_wait_read();  // shared memory must outlive the last bulk store's reads
     if (dead) {
         // a wait ran out: wait once more, with the limit, for whatever may still be on its way into the ring, so that

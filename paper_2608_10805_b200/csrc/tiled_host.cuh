@@ -128,8 +128,10 @@ inline wtconv_status launch_epilogue(const wtconv_desc *d, const wt::EpiloguePtr
     const int KK = d->k * d->k;
     size_t smem = sizeof(double) * (KK + 1 + (size_t)d->L * 4 * KK);
     // an ordinary launch: it starts when the kernels that produced the partial sums have completed
-    wt::unfold_epilogue_kernel<0><<<d->C, 128, smem, st>>>(d->C, d->k, d->L, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl,
-                                                        gsl);
+    // released by the last block of the kernel before it (or at that kernel's completion); waits for it itself
+    if (wt::launch_overlapped(wt::unfold_epilogue_kernel<0>, (unsigned)d->C, 128u, smem, st, d->C, d->k, d->L, ep, w0, s0, b0,
+                              wl, sl, gw0, gs0, gb0, gwl, gsl) != cudaSuccess)
+        return WTCONV_ERR_CUDA;
     return launch_status();
 }
 

@@ -825,51 +825,58 @@ unfold_epilogue_kernel(int C, int K, int L, EpiloguePtrs ep, const float *__rest
                        const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
                        const float *__restrict__ sl, float *__restrict__ dw0, float *__restrict__ ds0,
                        float *__restrict__ db0, float *__restrict__ dwl, float *__restrict__ dsl) {
-    extern __shared__ double folded[];  // [KK+1] base, then [L][4][KK]
+    extern __shared__ double prod[];  // dWfold[e] * W[e]: [KK+1] base (tap products, then dbfold * b), then [L][4][KK]
     const int c = blockIdx.x, KK = K * K;
     const int n0 = KK + 1, nl = 4 * KK;
     dependents_may_start();  // the next kernel on the stream may run its set-up beside this one
+    wait_for_predecessor();  // the partial sums come from the kernels before this one
     int written = 0x7fffffff;  // slots of this channel that hold sums
     if (ep.grp > 0) {
         const long long first_unit = (long long)(c / ep.grp) * ep.B;
         written = block_of_unit(first_unit + ep.B - 1, ep.nblocks, ep.units) - block_of_unit(first_unit, ep.nblocks, ep.units) + 1;
     }
+    // One entry per thread and pass: its partial sums, the parameter it meets in the scale gradient and its scale are
+    // all requested before the first is used, so the block pays one memory round trip.
     for (int e = threadIdx.x; e < n0 + L * nl; e += blockDim.x) {
-        double acc = 0.0;
+        const float *q;
+        size_t stride;
+        int n;
+        float wv, sv;
+        float *dst;
         if (e < n0) {
-            const float *q = ep.part0 + (size_t)c * ep.np0 * n0 + e;
-            const int n = ep.np0 < written ? ep.np0 : written;
-            for (int i = 0; i < n; ++i) acc += (double)q[(size_t)i * n0];
+            q = ep.part0 + (size_t)c * ep.np0 * n0 + e;
+            stride = n0;
+            n = ep.np0 < written ? ep.np0 : written;
+            wv = e < KK ? w0[(size_t)c * KK + e] : (b0 ? b0[c] : 0.f);
+            sv = s0[c];
+            dst = e < KK ? dw0 + (size_t)c * KK + e : (b0 ? db0 + c : nullptr);
         } else {
-            int l = (e - n0) / nl, t = (e - n0) - l * nl;
-            const float *q = ep.partl[l] + (size_t)c * ep.npl[l] * nl + t;
-            const int n = ep.npl[l] < written ? ep.npl[l] : written;
-            for (int i = 0; i < n; ++i) acc += (double)q[(size_t)i * nl];
+            const int l = (e - n0) / nl, t = (e - n0) - l * nl;
+            q = ep.partl[l] + (size_t)c * ep.npl[l] * nl + t;
+            stride = nl;
+            n = ep.npl[l] < written ? ep.npl[l] : written;
+            wv = wl[((size_t)l * C + c) * nl + t];
+            sv = sl[((size_t)l * C + c) * 4 + t / KK];
+            dst = dwl + ((size_t)l * C + c) * nl + t;
         }
-        folded[e] = acc;
+        double acc = 0.0;  // fixed slot order, fp64: the batch sum does not depend on the launch geometry's timing
+        for (int i = 0; i < n; ++i) acc += (double)q[(size_t)i * stride];
+        prod[e] = acc * (double)wv;
+        if (dst) *dst = (float)((double)sv * acc);  // Eq. 9: dW = s dWfold, db = s dbfold
     }
     __syncthreads();
-    const double s0c = (double)s0[c];
-    for (int t = threadIdx.x; t < KK; t += blockDim.x) dw0[(size_t)c * KK + t] = (float)(s0c * folded[t]);
-    for (int e = threadIdx.x; e < L * nl; e += blockDim.x) {
-        int l = e / nl, r = e - l * nl, sub = r / KK;
-        dwl[((size_t)l * C + c) * nl + r] = (float)((double)sl[((size_t)l * C + c) * 4 + sub] * folded[n0 + e]);
-    }
-    if (threadIdx.x == 0) {
+    // Eq. 9: ds = <dWfold, W> per class (+ dbfold b on the base class), terms added in index order
+    for (int cls = threadIdx.x; cls < 1 + 4 * L; cls += blockDim.x) {
         double a = 0.0;
-        for (int t = 0; t < KK; ++t) a += folded[t] * (double)w0[(size_t)c * KK + t];
-        if (b0) {
-            a += folded[KK] * (double)b0[c];
-            db0[c] = (float)(s0c * folded[KK]);
+        if (cls == 0) {
+            for (int t = 0; t < KK; ++t) a += prod[t];
+            if (b0) a += prod[KK];
+            ds0[c] = (float)a;
+        } else {
+            const double *pq = prod + n0 + (cls - 1) * KK;
+            for (int t = 0; t < KK; ++t) a += pq[t];
+            dsl[((size_t)((cls - 1) >> 2) * C + c) * 4 + ((cls - 1) & 3)] = (float)a;
         }
-        ds0[c] = (float)a;
-    }
-    for (int e = threadIdx.x + 1; e < 1 + L * 4; e += blockDim.x) {
-        int l = (e - 1) / 4, sub = (e - 1) & 3;
-        double a = 0.0;
-        const float *wq = wl + (((size_t)l * C + c) * 4 + sub) * KK;
-        for (int t = 0; t < KK; ++t) a += folded[n0 + l * nl + sub * KK + t] * (double)wq[t];
-        dsl[((size_t)l * C + c) * 4 + sub] = (float)a;
     }
 }
 
