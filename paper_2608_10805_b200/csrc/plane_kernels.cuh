@@ -1282,19 +1282,21 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             const int mytag = item.meta < 0 ? item.slot * 64 + cls : -1;
             scr[tid * (KK + 2) + KK + 1] = __int_as_float(mytag);
             __syncthreads();
-            // the threads of one (plane, class) are neighbours in the item list: note where each run starts
-            int *run_start = reinterpret_cast<int *>(scr + nthr * (KK + 2));
-            if (mytag >= 0 && (tid == 0 || __float_as_int(scr[(tid - 1) * (KK + 2) + KK + 1]) != mytag))
-                run_start[item.slot * ncls + cls] = tid;
+            // the threads of one (plane, class) are neighbours in the item list: note where each run starts and ends
+            int *run_start = reinterpret_cast<int *>(scr + nthr * (KK + 2)), *run_end = run_start + g.NPL * ncls;
+            if (mytag >= 0) {
+                if (tid == 0 || __float_as_int(scr[(tid - 1) * (KK + 2) + KK + 1]) != mytag) run_start[item.slot * ncls + cls] = tid;
+                if (tid == nthr - 1 || __float_as_int(scr[(tid + 1) * (KK + 2) + KK + 1]) != mytag) run_end[item.slot * ncls + cls] = tid + 1;
+            }
             __syncthreads();
             const int slotp = blockIdx.x - block_of_unit((long long)cg * g.B, gridDim.x, g.units);
             for (int e = tid; e < nvalid * ncls * (KK + 1); e += nthr) {
                 const int sc = e / (KK + 1), t = e - sc * (KK + 1), slot = sc / ncls, c2 = sc - slot * ncls;
                 if (c2 > 0 && t == KK) continue;
-                const int tag = slot * 64 + c2, ch = c + slot;
+                const int ch = c + slot;
                 float sacc = 0.f;
-                for (int th = run_start[sc]; th < nthr && __float_as_int(scr[th * (KK + 2) + KK + 1]) == tag; ++th)
-                    sacc += scr[th * (KK + 2) + t];
+                const int th1 = run_end[sc];  // known trip count: the loads of the sum do not wait for one another
+                for (int th = run_start[sc]; th < th1; ++th) sacc += scr[th * (KK + 2) + t];
                 if (c2 == 0) {
                     part0[((size_t)ch * g.np + slotp) * (KK + 1) + t] = sacc;
                 } else {
@@ -1303,8 +1305,11 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 }
             }
             __syncthreads();
-            for (int i = tid; i < g.wtab_off / 4; i += nthr)  // restore the zero halos of the arrays
-                reinterpret_cast<float4 *>(sm)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            {   // restore the zero halos under the scratch (the rest of the arrays was not touched)
+                int nz = (nthr * (KK + 2) + 2 * g.NPL * ncls + 3) / 4;
+                if (nz > g.wtab_off / 4) nz = g.wtab_off / 4;
+                for (int i = tid; i < nz; i += nthr) reinterpret_cast<float4 *>(sm)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
             for (int t = 0; t < KK; ++t) accw[t] = 0.f;
             gsum = 0.f;
@@ -1580,7 +1585,7 @@ inline bool plan_bwd_fused_th(int B, int C, int H, int W, int L, int elem_bytes,
         const int wtab = npl * (1 + 4 * L) * WT_STRIDE;
         const int T = (npl * M + 31) & ~31;
         long long arrays = (long long)npl * slot;
-        const long long scratch = (long long)T * (KK + 2) + (long long)npl * (1 + 4 * L);  // flush scratch: sums, tags, run starts
+        const long long scratch = (long long)T * (KK + 2) + 2LL * npl * (1 + 4 * L);  // flush scratch: sums, tags, run starts and ends
         if (scratch > arrays) arrays = scratch;
         const bool can_bulk = (C % npl == 0) && (((long long)npl * g.plane_bytes) % 16 == 0) && !((tune >> 20) & 1);
         bool any = false;
