@@ -71,6 +71,7 @@ def run_gpu(wl, I, flags=0, guarded=True):
     wsg = Guarded(max(fb, bb, 256))
     bands.append(wsg)
     ws = wsg.body
+    ws.fill_(0xFF)  # NaN as floats, -1 as words: a call that depends on what it finds in its workspace shows
     flags_h = torch.zeros(2, dtype=torch.int32).pin_memory()
     wt.wtconv_forward(desc, x, w0, s0, b0, wl_, sl, out, ws)
     wt.wtconv_read_status(desc, ws, flags_h[0:1])

@@ -61,3 +61,38 @@ def test_autograd_layer_reports_an_earlier_timeout():
         ag.status_watch.after_call(desc, ws)
         ag.status_watch.drain()
     ag.status_watch.drain()  # nothing is left pending
+
+
+def test_a_workspace_carries_nothing_from_one_call_to_the_next():
+    """No call clears its workspace.  A call that timed out leaves its tag in the status words and its partial
+    sums (of another shape) in the workspace; a later call of a different shape on the same workspace must read as
+    clean and give the oracle's results."""
+    first, flags1 = CASES[0]
+    second = Workload("plane_14_after", 4, 24, 14, 14, 5, 2, "f32", 73)
+    tdt1, tdt2 = wt.DTYPE_NAMES[first.dtype], wt.DTYPE_NAMES[second.dtype]
+    bad = wt.make_desc(first.B, first.C, first.H, first.W, first.k, first.L, tdt1, flags1 | wt.FLAG_TEST_NO_COPY)
+    good = wt.make_desc(second.B, second.C, second.H, second.W, second.k, second.L, tdt2, wt.FLAG_NO_TEAM)
+    assert wt.wtconv_plan_name(good) == "plane"
+    nbytes = max(max(wt.wtconv_workspace_bytes(bad)), max(wt.wtconv_workspace_bytes(good)))
+    ws = torch.full((nbytes,), 0xFF, dtype=torch.uint8, device="cuda")
+    flag = torch.zeros(3, dtype=torch.int32).pin_memory()
+    I1, I2 = inputs.make_inputs(first), inputs.make_inputs(second)
+    x1, g1 = to_dev(I1["x"], tdt1), to_dev(I1["g"], tdt1)
+    p1 = [to_dev(I1[k]) for k in ("w0", "s0", "wl", "sl")]
+    gx1 = torch.empty_like(x1)
+    gp1 = [torch.empty_like(t) for t in p1]
+    wt.wtconv_backward(bad, x1, g1, p1[0], p1[1], None, p1[2], p1[3], gx1, gp1[0], gp1[1], None, gp1[2], gp1[3], ws)
+    wt.wtconv_read_status(bad, ws, flag[0:1])
+    x2, g2 = to_dev(I2["x"], tdt2), to_dev(I2["g"], tdt2)
+    p2 = [to_dev(I2[k]) for k in ("w0", "s0", "wl", "sl")]
+    out2, gx2 = torch.full_like(x2, float("nan")), torch.full_like(x2, float("nan"))
+    gp2 = [torch.full_like(t, float("nan")) for t in p2]
+    wt.wtconv_forward(good, x2, p2[0], p2[1], None, p2[2], p2[3], out2, ws)
+    wt.wtconv_read_status(good, ws, flag[1:2])
+    wt.wtconv_backward(good, x2, g2, p2[0], p2[1], None, p2[2], p2[3], gx2, gp2[0], gp2[1], None, gp2[2], gp2[3], ws)
+    wt.wtconv_read_status(good, ws, flag[2:3])
+    torch.cuda.synchronize()
+    assert int(flag[0]) != 0 and int(flag[1]) == 0 and int(flag[2]) == 0
+    f = lambda t: t.double().cpu().numpy()
+    got = (f(out2), dict(dx=f(gx2), dw0=f(gp2[0]), ds0=f(gp2[1]), db0=None, dwl=f(gp2[2]), dsl=f(gp2[3])))
+    assert_close(second, got, run_oracle(second, I2))
