@@ -163,7 +163,7 @@ wtconv_status wtconv_backward(const wtconv_desc *desc, const void *x, const void
 
 /* Device-side status of the last call that used `workspace` (device pointer; NULL = the array built into the
  * library that wtconv_backward_static uses, on the current device) with this descriptor: enqueues on
- * `stream` a one-thread kernel that evaluates the workspace's status words and a copy of the verdict into
+ * `stream` a one-thread kernel that evaluates the workspace's status words and a copy of the result into
  * *h_flag (a HOST int32, pinned if the copy is to be asynchronous).  Once the stream has reached this point, 0
  * means every bounded wait inside the kernels completed (the paper's kernels wait for nothing; ours wait only
  * for their own bulk copies); non-zero means a wait ran out and the outputs of that call are not valid (report

@@ -630,7 +630,7 @@ wtconv_status wtconv_read_status(const wtconv_desc *d, void *workspace, int32_t 
         return WTCONV_OK;
     }
     // the status words open every workspace the plane kernels use: compare the timeout tag with the tag of the
-    // last launch on the device, then fetch the verdict
+    // last launch on the device, then fetch the result
     int *words = (int *)workspace;
     resolve_status_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(words);
     if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
