@@ -124,10 +124,76 @@ bool use_window_path(const wtconv_desc *d) {
     return wt::window::supported(d->B, d->C, d->H, d->W, d->k, d->L, d->dtype);
 }
 
+// k = 3 through the k = 5 kernels.  A 3 x 3 depthwise kernel is a 5 x 5 kernel with a border of zeros, so wherever the
+// kernels that keep planes on chip (k = 5 only) serve the shape, the parameters are copied into 5 x 5 tables at the
+// head of the workspace, the k = 5 path runs on them, and the backward copies the inner 3 x 3 of the 5 x 5 weight
+// gradients out (the border's gradients are dropped; the scale and bias gradients are unaffected, since the border
+// weights are zero).  16 of 25 taps multiply zeros, and it is still 2-3 x faster than the per-level kernels.
+wtconv_desc as_k5(const wtconv_desc *d) {
+    wtconv_desc d5 = *d;
+    d5.k = 5;
+    return d5;
+}
+bool use_k3_embedding(const wtconv_desc *d) {
+    if (d->k != 3 || (d->flags & (WTCONV_FLAG_TILED_ONLY | WTCONV_FLAG_REFERENCE_CHAIN))) return false;
+    const wtconv_desc d5 = as_k5(d);
+    return use_plane_path(&d5) || use_window_path(&d5);
+}
+// Workspace head of the embedding: w0 [C][25], wl [L][C][4][25], then the same two for the gradients; the k = 5
+// path's own workspace follows.
+struct EmbedLayout {
+    size_t w0, wl, gw0, gwl, inner;  // byte offsets
+    size_t nf0, nfl;                 // filters in w0 / wl
+};
+EmbedLayout embed_layout(const wtconv_desc *d) {
+    EmbedLayout e;
+    e.nf0 = (size_t)d->C;
+    e.nfl = (size_t)d->L * d->C * 4;
+    e.w0 = 0;
+    e.wl = align_up(e.w0 + e.nf0 * 25 * sizeof(float));
+    e.gw0 = align_up(e.wl + e.nfl * 25 * sizeof(float));
+    e.gwl = align_up(e.gw0 + e.nf0 * 25 * sizeof(float));
+    e.inner = align_up(e.gwl + e.nfl * 25 * sizeof(float));
+    return e;
+}
+// filters [nf0] of a and [nfl] of b, 3 x 3 -> 5 x 5 with a zero border
+__global__ void embed_k3_kernel(const float *__restrict__ a, const float *__restrict__ b, float *__restrict__ ae,
+                                float *__restrict__ be, size_t nf0, size_t nfl) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (nf0 + nfl) * 25) return;
+    const size_t f = i / 25;
+    const int t = (int)(i - f * 25), u = t / 5, v = t - u * 5;
+    const bool inner = u >= 1 && u <= 3 && v >= 1 && v <= 3;
+    const int t3 = (u - 1) * 3 + (v - 1);
+    if (f < nf0) ae[f * 25 + t] = inner ? a[f * 9 + t3] : 0.f;
+    else be[(f - nf0) * 25 + t] = inner ? b[(f - nf0) * 9 + t3] : 0.f;
+}
+// the inner 3 x 3 of 5 x 5 gradients
+__global__ void extract_k3_kernel(const float *__restrict__ ae, const float *__restrict__ be, float *__restrict__ a,
+                                  float *__restrict__ b, size_t nf0, size_t nfl) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (nf0 + nfl) * 9) return;
+    const size_t f = i / 9;
+    const int t = (int)(i - f * 9), u = t / 3 + 1, v = t - (t / 3) * 3 + 1;
+    if (f < nf0) a[f * 9 + t] = ae[f * 25 + u * 5 + v];
+    else b[(f - nf0) * 9 + t] = be[(f - nf0) * 25 + u * 5 + v];
+}
+
 template <typename T, int K>
 wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, const float *s0, const float *b0,
                          const float *wl, const float *sl, void *out, char *ws, cudaStream_t st) {
     if (use_ref_chain(d)) return wt::refchain::forward<T, K>(d, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st);
+    if constexpr (K == 3) {
+        if (use_k3_embedding(d)) {
+            const wtconv_desc d5 = as_k5(d);
+            const EmbedLayout e = embed_layout(d);
+            float *w0e = (float *)(ws + e.w0), *wle = (float *)(ws + e.wl);
+            const size_t n = (e.nf0 + e.nfl) * 25;
+            embed_k3_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w0, wl, w0e, wle, e.nf0, e.nfl);
+            if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
+            return forward_tk<T, 5>(&d5, x, w0e, s0, b0, wle, sl, out, ws + e.inner, st);
+        }
+    }
     if constexpr (K == 5) {
         if (use_team_path(d))
             return wt::team::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st,
@@ -161,6 +227,20 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
     if (use_ref_chain(d))
         return wt::refchain::backward<T, K>(d, (const T *)x, (const T *)g, w0, s0, b0, wl, sl, (T *)gx, gw0, gs0, gb0, gwl, gsl,
                                             ws, st);
+    if constexpr (K == 3) {
+        if (use_k3_embedding(d)) {
+            const wtconv_desc d5 = as_k5(d);
+            const EmbedLayout e = embed_layout(d);
+            float *w0e = (float *)(ws + e.w0), *wle = (float *)(ws + e.wl), *gw0e = (float *)(ws + e.gw0), *gwle = (float *)(ws + e.gwl);
+            const size_t n = (e.nf0 + e.nfl) * 25, n3 = (e.nf0 + e.nfl) * 9;
+            embed_k3_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w0, wl, w0e, wle, e.nf0, e.nfl);
+            if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
+            const wtconv_status st5 = backward_tk<T, 5>(&d5, x, g, w0e, s0, b0, wle, sl, gx, gw0e, gs0, gb0, gwle, gsl, ws + e.inner, st);
+            if (st5 != WTCONV_OK) return st5;
+            extract_k3_kernel<<<(unsigned)((n3 + 255) / 256), 256, 0, st>>>(gw0e, gwle, gw0, gwl, e.nf0, e.nfl);
+            return launch_status();
+        }
+    }
     if constexpr (K == 5) {
         if (use_team_path(d)) {
             wt::EpiloguePtrs ep = {};
@@ -211,12 +291,20 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
     } while (0)
 
 size_t fwd_ws_bytes(const wtconv_desc *d) {
+    if (use_k3_embedding(d)) {
+        const wtconv_desc d5 = as_k5(d);
+        return embed_layout(d).inner + fwd_ws_bytes(&d5);
+    }
     if (use_ref_chain(d)) return wt::refchain::make_plan(d).fwd_bytes;
     if (use_plane_path(d)) return align_up(wt::plane::forward_workspace_bytes(d->B, d->C, d->H, d->W, d->L));
     if (use_window_path(d)) return align_up(wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).fwd_bytes);
     return make_tiled_plan(d).fwd_bytes;
 }
 size_t bwd_ws_bytes(const wtconv_desc *d) {
+    if (use_k3_embedding(d)) {
+        const wtconv_desc d5 = as_k5(d);
+        return embed_layout(d).inner + bwd_ws_bytes(&d5);
+    }
     if (use_ref_chain(d)) return wt::refchain::make_plan(d).bwd_bytes;
     if (use_team_path(d)) return align_up(wt::team::backward_workspace_bytes(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), team_force_g(d)));
     if (use_window_path(d)) return align_up(wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).bwd_bytes);
@@ -349,6 +437,10 @@ wtconv_status wtconv_workspace_bytes(const wtconv_desc *d, size_t *fwd_bytes, si
 
 const char *wtconv_plan_name(const wtconv_desc *d) {
     if (validate_desc(d) != WTCONV_OK) return nullptr;
+    if (use_k3_embedding(d)) {  // the kernels that run: the k = 5 path's
+        const wtconv_desc d5 = as_k5(d);
+        return wtconv_plan_name(&d5);
+    }
     return use_ref_chain(d) ? "reference-chain" : use_team_path(d) ? "team" : use_plane_path(d) ? "plane" : use_window_path(d) ? "window" : "tiled";
 }
 
@@ -357,6 +449,11 @@ wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
     if (st != WTCONV_OK) return st;
     if (!buf || n == 0) return WTCONV_ERR_NULL;
     buf[0] = 0;
+    if (use_k3_embedding(d)) {
+        const wtconv_desc d5 = as_k5(d);
+        const int o = snprintf(buf, n, "3x3 kernels in 5x5 tables: ");
+        return o > 0 && (size_t)o < n ? wtconv_plan_describe(&d5, buf + o, n - o) : WTCONV_OK;
+    }
     if (use_ref_chain(d))
         snprintf(buf, n, "reference-chain (separate operators, intermediates in HBM)%s%s",
                  (d->flags & WTCONV_FLAG_ABLATE_FUSED_ANALYSIS) ? " +fused-analysis" : "",
@@ -380,6 +477,13 @@ wtconv_status wtconv_plan_describe(const wtconv_desc *d, char *buf, size_t n) {
 wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *bwd) {
     wtconv_status st = validate_desc(d);
     if (st != WTCONV_OK) return st;
+    if (use_k3_embedding(d)) {  // the k = 5 path's launches + the table kernel (+ the gradient copy in the backward)
+        const wtconv_desc d5 = as_k5(d);
+        st = wtconv_launch_count(&d5, fwd, bwd);
+        if (st == WTCONV_OK && fwd) *fwd += 1;
+        if (st == WTCONV_OK && bwd) *bwd += 2;
+        return st;
+    }
     if (use_ref_chain(d)) {
         const bool fa = d->flags & WTCONV_FLAG_ABLATE_FUSED_ANALYSIS, cs = d->flags & WTCONV_FLAG_ABLATE_COLLAPSED_SYNTHESIS;
         const int nf = (fa ? 1 : 0) + d->L * (fa ? 2 : 3) + (d->L > 1 && !fa ? d->L - 1 : 0) + 2 + (cs ? 1 : 2 * d->L + 1);
@@ -623,6 +727,12 @@ wtconv_status wtconv_read_status(const wtconv_desc *d, void *workspace, int32_t 
         workspace = scratch;
     }
     if ((uintptr_t)workspace & (ALIGN - 1)) return WTCONV_ERR_ALIGNMENT;
+    wtconv_desc d5;
+    if (use_k3_embedding(d)) {  // the status words belong to the k = 5 path, behind the parameter tables
+        workspace = (char *)workspace + embed_layout(d).inner;
+        d5 = as_k5(d);
+        d = &d5;
+    }
     if (use_window_path(d) && d->L > 2)  // the carrier's whole-plane kernels keep the only status word of this path
         workspace = (char *)workspace + wt::window::ws_plan(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype)).deep;
     else if (!use_plane_path(d)) {  // the tiled, window (L <= 2) and reference kernels wait for nothing and keep no status word

@@ -78,9 +78,13 @@ def test_wtconvnext_depth_schedule_bf16(name):
     _run_full_and_compare(wl)
 
 
-@pytest.mark.parametrize("name", ["stage1_k3_f32", "stage1_k7_f32"])
-def test_kernel_size_variants(name):
-    _run_full_and_compare(inputs.WORKLOADS[name])
+@pytest.mark.parametrize("name,flags", [("stage1_k3_f32", 0), ("stage1_k3_f32", wt.FLAG_TILED_ONLY), ("stage1_k7_f32", 0)],
+                         ids=["k3_in_5x5_tables", "k3_per_level_kernels", "k7"])
+def test_kernel_size_variants(name, flags):
+    wl = inputs.WORKLOADS[name]
+    plan = wt.wtconv_plan_name(wt.make_desc(wl.B, wl.C, wl.H, wl.W, wl.k, wl.L, wt.DTYPE_NAMES[wl.dtype], flags))
+    assert plan == ("plane" if (wl.k == 3 and flags == 0) else "tiled")  # 3 x 3 kernels ride the k = 5 kernels by default
+    _run_full_and_compare(wl, flags=flags)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "f16"])

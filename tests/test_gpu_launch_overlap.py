@@ -18,7 +18,7 @@ LAYERS = [Workload("ov_plane_28", 6, 24, 28, 28, 5, 2, "bf16", 81),   # fused ba
           Workload("ov_team_7", 12, 32, 7, 7, 5, 1, "bf16", 82),      # team kernels
           Workload("ov_split_40", 3, 10, 40, 36, 5, 3, "f32", 83),    # split backward (weight-gradient + input-gradient kernels)
           Workload("ov_plane_14", 8, 40, 14, 14, 5, 1, "f16", 84),
-          Workload("ov_tiled_k3", 2, 6, 20, 24, 3, 2, "f32", 85)]     # per-level kernels between the persistent ones
+          Workload("ov_tiled_k7", 2, 6, 20, 24, 7, 2, "f32", 85)]     # per-level kernels between the persistent ones
 
 
 def test_layers_share_one_workspace_back_to_back():
