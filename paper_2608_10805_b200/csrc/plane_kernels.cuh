@@ -27,6 +27,10 @@
 //    rotated-kernel convolution, synthesis and store on the same window.  Shapes whose tiles do not fit
 //    one pass of 256 threads take the split pair instead: a weight-gradient kernel with class-major
 //    thread allocation plus the FLIP instantiation of the forward kernel.
+//  * Launches overlap: every kernel here is started with programmatic stream serialisation (common.cuh), does its
+//    set-up in shared memory and registers beside the tail of the kernel before it and only then waits for that
+//    kernel; no call puts a clearing operation between two kernels (status words are tagged per call, the epilogue
+//    is told which partial-sum slots the blocks write).
 //  * Host side: plans (threads, blocks per SM, planes per unit, tile height, ring depth) come from a
 //    search over a small cost model and are cached per shape.
 #pragma once

@@ -495,12 +495,12 @@ wtconv_status wtconv_launch_count(const wtconv_desc *d, int32_t *fwd, int32_t *b
         if (bwd) *bwd = d->L > 2 ? 7 : 2;
     } else if (use_team_path(d)) {
         if (fwd) *fwd = 1;
-        if (bwd) *bwd = 2;  // fused backward + epilogue (plus one memset node)
+        if (bwd) *bwd = 2;  // fused backward + epilogue (and nothing else on the stream)
     } else if (use_plane_path(d)) {
         if (fwd) *fwd = 1;
         if (bwd) {
             wt::plane::Geom gq;
-            /* fused backward + epilogue, or weight-gradient + input-gradient + epilogue (plus one memset node) */
+            /* fused backward + epilogue, or weight-gradient + input-gradient + epilogue (and nothing else on the stream) */
             *bwd = wt::plane::plan_bwd_fused(d->B, d->C, d->H, d->W, d->L, (int)elem_bytes(d->dtype), gq, d->flags >> 8) ? 2 : 3;
         }
     } else {
