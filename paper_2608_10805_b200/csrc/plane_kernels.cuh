@@ -1125,12 +1125,12 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
     const int cls = (item.meta >> 24) & 0x3f;
     // No barrier separates a unit's synthesis (which reads only Z and registers) from the next unit's staging.
     // With the planes already in shared memory (BULK == 2) the staging is left to the whole warps that hold
-    // level tiles only, two patches each if need be, while the base-tile threads finish the synthesis.  With
-    // staging from global memory every thread takes part: two patches per thread would make the exposed
-    // load-to-store chain twice as long (measured slower at 56 x 56 fp32).
+    // level tiles only while the base-tile threads finish the synthesis - as long as one patch each covers the
+    // unit.  Otherwise every thread takes part: two patches per thread make the exposed load-to-store chain twice
+    // as long (measured slower at 56 x 56, from global memory as well as from the ring).
     int nstagers = (nlevel_items / 32) * 32;
     if (nstagers > nthr) nstagers = nthr;
-    if (BULK != 2 || nstagers * 4 < nthr || g.NPL * g.npatch4 > 2 * nstagers) nstagers = nthr;
+    if (BULK != 2 || nstagers * 4 < nthr || g.NPL * g.npatch4 > nstagers) nstagers = nthr;
     const int srank = tid < nstagers ? tid : 0x3fffffff;
     const bool hoist_patch = g.vec && L >= 2 && g.NPL * g.npatch4 <= 2 * nstagers;
     const PatchD patch0 = decode_patch(g, g.offA, hoist_patch ? srank : 0x3fffffff);
