@@ -623,9 +623,11 @@ __device__ __forceinline__ void stage_level(float *sm, const Geom &g, const int 
 // 4-column x TH-row output tile of a 5x5 correlation.  `src` = array + (TH*ty)*pitch + 4*tx is the
 // window's top-left element (the array's halo of 2 makes window row rr = output row + tap row), 16-byte
 // aligned; eight floats per window row.
-template <int TH>
+// KEEP: the window's interior (rows 2 .. TH+1, columns 2 .. 5: the tile's own elements) is copied to `keep` on the
+// way through the registers.
+template <int TH, bool KEEP = false>
 __device__ __forceinline__ void conv_tile(const float *__restrict__ src, int pitch, const float (&w)[KK],
-                                          float (&acc)[TH][4]) {
+                                          float (&acc)[TH][4], float (*keep)[4] = nullptr) {
 #pragma unroll
     for (int r = 0; r < TH; ++r)
 #pragma unroll
@@ -636,6 +638,10 @@ __device__ __forceinline__ void conv_tile(const float *__restrict__ src, int pit
 #pragma unroll
     for (int rr = 0; rr < TH + 4; ++rr) {
         const float in[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+        if (KEEP && rr >= 2 && rr < TH + 2) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) keep[rr - 2][c] = in[c + 2];
+        }
         if (rr + 1 < TH + 4) {
             n0 = *reinterpret_cast<const float4 *>(src + (rr + 1) * pitch);
             n1 = *reinterpret_cast<const float4 *>(src + (rr + 1) * pitch + 4);
@@ -1212,15 +1218,24 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             const int pitch = item.meta & 0x3ff;
             const float *ysrc = sm + item.src;            // Y window (x side)
             const float *gsrc = sm + item.src + item.dg;  // D window (grad_out side)
-            {
-                // weight gradient: the tile's D values are the window's interior
-                float d[TH][4];
+            // With 4-row tiles the registers allow the rotated convolution to go first and to hand the tile's D values
+            // (the interior of the window it reads anyway) to the weight-gradient taps; with 8-row tiles the D values
+            // are loaded on their own.
+            float d[TH][4];
+            if (TH == 4) {
+                float w[KK];
+                load_weights(sm + item.wt, w);
+                conv_tile<TH, true>(gsrc, pitch, w, acc, d);
+            } else {
 #pragma unroll
                 for (int rr = 0; rr < TH; ++rr) {
                     const float2 q0 = *reinterpret_cast<const float2 *>(gsrc + (rr + 2) * pitch + 2);
                     const float2 q1 = *reinterpret_cast<const float2 *>(gsrc + (rr + 2) * pitch + 4);
                     d[rr][0] = q0.x; d[rr][1] = q0.y; d[rr][2] = q1.x; d[rr][3] = q1.y;
                 }
+            }
+            {
+                // weight gradient: the tile's D values are the window's interior
                 if (cls == 0) {
 #pragma unroll
                     for (int rr = 0; rr < TH; ++rr)
@@ -1249,10 +1264,11 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                     }
                 }
             }
-            // input gradient: rotated-kernel conv of the D window
-            float w[KK];
-            load_weights(sm + item.wt, w);
-            conv_tile<TH>(gsrc, pitch, w, acc);
+            if (TH != 4) {  // input gradient: rotated-kernel conv of the D window
+                float w[KK];
+                load_weights(sm + item.wt, w);
+                conv_tile<TH>(gsrc, pitch, w, acc);
+            }
             if (item.z >= 0) {
                 const int zp = (item.meta >> 10) & 0x3ff, zleft = (item.meta >> 20) & 0xf;
                 float *z = sm + item.z;
