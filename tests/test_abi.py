@@ -85,7 +85,19 @@ def test_plan_and_launch_count(lib):
     assert wt.wtconv_launch_count(dn) == (4, 5)
     dt = wt.make_desc(2, 3, 56, 56, 5, 3, "f32", wt.FLAG_TILED_ONLY)
     assert wt.wtconv_plan_name(dt) == "tiled"
-    assert wt.wtconv_plan_name(wt.make_desc(2, 3, 56, 56, 7, 3, "f32")) == "tiled"  # k = 3 / 7: tiled kernels
+    assert wt.wtconv_plan_name(wt.make_desc(2, 3, 56, 56, 7, 3, "f32")) == "tiled"  # k = 7: per-level kernels
+    # k = 3 rides the k = 5 kernels (filters in zero-bordered 5 x 5 tables: one launch more forward, two backward,
+    # the tables at the head of the workspace) unless the per-level kernels are asked for
+    d3, d5 = wt.make_desc(2, 8, 56, 56, 3, 3, "f32"), wt.make_desc(2, 8, 56, 56, 5, 3, "f32")
+    assert wt.wtconv_plan_name(d3) == wt.wtconv_plan_name(d5) == "plane"
+    f5, b5 = wt.wtconv_launch_count(d5)
+    assert wt.wtconv_launch_count(d3) == (f5 + 1, b5 + 2)
+    tables = 2 * (8 * 25 * 4 + 3 * 8 * 4 * 25 * 4)  # parameters and their gradients, before 256-byte rounding
+    w3, w5 = wt.wtconv_workspace_bytes(d3), wt.wtconv_workspace_bytes(d5)
+    assert tables <= w3[0] - w5[0] <= tables + 4 * 256 and w3[1] - w5[1] == w3[0] - w5[0]
+    assert wt.wtconv_plan_describe(d3).startswith("3x3 kernels in 5x5 tables: plane")
+    d3t = wt.make_desc(2, 8, 56, 56, 3, 3, "f32", wt.FLAG_TILED_ONLY)
+    assert wt.wtconv_plan_name(d3t) == "tiled" and wt.wtconv_launch_count(d3t) == (4, 5)
 
 
 def test_scratch_memory_accounting(lib):
