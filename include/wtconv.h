@@ -75,7 +75,8 @@ typedef enum {
  * kernels: by default a k = 3 layer whose shape the plane-resident k = 5 kernels serve is run through them with its
  * 3 x 3 filters copied into zero-bordered 5 x 5 tables at the head of the workspace (one small launch more per call,
  * two in the backward, which copies the inner 3 x 3 of the 5 x 5 weight gradients out; results are those of the
- * 3 x 3 layer exactly as defined, the border taps multiply zeros). */
+ * 3 x 3 layer exactly as defined; the block-per-plane kernels skip the border taps, the team and window kernels
+ * multiply them with zeros). */
 #define WTCONV_FLAG_TILED_ONLY 1u
 /* Test aid for the timeout path of the bounded device-side waits: no bulk copy is issued at all and the wait
  * limit is tiny, so every wait for a copy runs out; the kernels record it in the status word and return

@@ -1,4 +1,5 @@
-// Whole-plane WTConv kernels for sm_100a (k = 5): every (b, c) plane's entire decomposition lives
+// Whole-plane WTConv kernels for sm_100a (k = 5, and k = 3 as the inner taps of 5 x 5 tables: KT = 3 builds of the
+// kernels leave the zero border out of the tap loops): every (b, c) plane's entire decomposition lives
 // in shared memory, so the only HBM traffic is the compulsory one (read x, write out; in the backward
 // read x and grad_out, write grad_x).
 //
@@ -134,6 +135,7 @@ struct Geom {
     int vec;                               // 1: W % 4 == 0, rows are staged with 4-element vector loads
     int no_copy;                           // test mode: bulk copies are never issued and waits give up quickly (the timeout path)
     unsigned tag;                          // non-zero tag of the call this launch belongs to (status words, see common.cuh)
+    int taps;                              // taps per side in use: 5, or 3 for 3 x 3 kernels in the middle of 5 x 5 tables
     int bulk;                              // 1: planes are fetched ahead with cp.async.bulk into a ring of raw buffers at raw_off
     int nstage, stage_bytes;               // ring depth (units in flight) and bytes per ring entry
     int raw_off, raw_slot_bytes, plane_bytes;  // raw staging buffer (float offset), bytes per plane slot / per plane
@@ -624,36 +626,66 @@ __device__ __forceinline__ void stage_level(float *sm, const Geom &g, const int 
 // window's top-left element (the array's halo of 2 makes window row rr = output row + tap row), 16-byte
 // aligned; eight floats per window row.
 // KEEP: the window's interior (rows 2 .. TH+1, columns 2 .. 5: the tile's own elements) is copied to `keep` on the
-// way through the registers.
-template <int TH, bool KEEP = false>
+// way through the registers.  KT: taps per side that are in use, 5 or 3 - a 3 x 3 kernel sits in the middle of the
+// 5 x 5 table and of the 5 x 5 window, its zero border is neither read nor multiplied.
+template <int TH, bool KEEP = false, int KT = 5>
 __device__ __forceinline__ void conv_tile(const float *__restrict__ src, int pitch, const float (&w)[KK],
                                           float (&acc)[TH][4], float (*keep)[4] = nullptr) {
+    constexpr int T0 = (5 - KT) / 2, T1 = 5 - T0;  // taps T0 .. T1-1 per side; window rows T0 .. TH+3-T0
 #pragma unroll
     for (int r = 0; r < TH; ++r)
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
     // the next window row is fetched while the current one is being used (software pipelining by hand)
-    float4 n0 = *reinterpret_cast<const float4 *>(src);
-    float4 n1 = *reinterpret_cast<const float4 *>(src + 4);
+    float4 n0 = *reinterpret_cast<const float4 *>(src + T0 * pitch);
+    float4 n1 = *reinterpret_cast<const float4 *>(src + T0 * pitch + 4);
 #pragma unroll
-    for (int rr = 0; rr < TH + 4; ++rr) {
+    for (int rr = T0; rr < TH + 4 - T0; ++rr) {
         const float in[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
         if (KEEP && rr >= 2 && rr < TH + 2) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) keep[rr - 2][c] = in[c + 2];
         }
-        if (rr + 1 < TH + 4) {
+        if (rr + 1 < TH + 4 - T0) {
             n0 = *reinterpret_cast<const float4 *>(src + (rr + 1) * pitch);
             n1 = *reinterpret_cast<const float4 *>(src + (rr + 1) * pitch + 4);
         }
 #pragma unroll
-        for (int u = 0; u < 5; ++u) {
+        for (int u = T0; u < T1; ++u) {
             const int r = rr - u;
             if (r >= 0 && r < TH) {
 #pragma unroll
-                for (int v = 0; v < 5; ++v)
+                for (int v = T0; v < T1; ++v)
 #pragma unroll
                     for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(w[u * 5 + v], in[c + v], acc[r][c]);
+            }
+        }
+    }
+}
+
+// The weight-gradient taps of one tile: accw[u][v] += sum over the tile of D[r][c] * Y[r + u][c + v] (window
+// coordinates; `d` = the tile's D values, `ysrc` = the window's top-left element).
+template <int TH, int KT>
+__device__ __forceinline__ void wgrad_taps(const float *__restrict__ ysrc, int pitch, const float (&d)[TH][4], float (&accw)[KK]) {
+    constexpr int T0 = (5 - KT) / 2, T1 = 5 - T0;
+    // the next window row is fetched while the current one is used
+    float4 n0 = *reinterpret_cast<const float4 *>(ysrc + T0 * pitch);
+    float4 n1 = *reinterpret_cast<const float4 *>(ysrc + T0 * pitch + 4);
+#pragma unroll
+    for (int rr = T0; rr < TH + 4 - T0; ++rr) {
+        const float in[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+        if (rr + 1 < TH + 4 - T0) {
+            n0 = *reinterpret_cast<const float4 *>(ysrc + (rr + 1) * pitch);
+            n1 = *reinterpret_cast<const float4 *>(ysrc + (rr + 1) * pitch + 4);
+        }
+#pragma unroll
+        for (int uu = T0; uu < T1; ++uu) {
+            const int dr = rr - uu;
+            if (dr >= 0 && dr < TH) {
+#pragma unroll
+                for (int v = T0; v < T1; ++v)
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) accw[uu * 5 + v] = fmaf(d[dr][cc], in[cc + v], accw[uu * 5 + v]);
             }
         }
     }
@@ -792,7 +824,7 @@ __device__ __forceinline__ void synth_block(const float *S, const Geom &g, int t
 
 // FLIP = false: out = WTConv(x).  FLIP = true: the same dataflow on grad_out with every kernel rotated
 // by 180 degrees and no bias gives grad_x.  MINB = resident blocks per SM the register budget is sized for.
-template <typename T, bool FLIP, int MAXT, int MINB, int TH>
+template <typename T, bool FLIP, int MAXT, int MINB, int TH, int KT>
 __global__ void __launch_bounds__(MAXT, MINB)
 plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const float *__restrict__ w0,
                  const float *__restrict__ s0, const float *__restrict__ b0, const float *__restrict__ wl,
@@ -921,7 +953,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
                 if (d.meta < 0) {
                     float w[KK];
                     load_weights(sm + d.wt, w);
-                    conv_tile<TH>(sm + d.src, d.meta & 0x3ff, w, acc);
+                    conv_tile<TH, false, KT>(sm + d.src, d.meta & 0x3ff, w, acc);
                     if (d.z >= 0) {
                         const int zp = (d.meta >> 10) & 0x3ff, zleft = (d.meta >> 20) & 0xf;
                         float *z = sm + d.z;
@@ -957,7 +989,7 @@ plane_fwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 // dWfold^l[u,v] += sum_{i,j} D^l[i,j] Y^l[i+u-2, j+v-2] (and the base class with grad_out and x), Sec. 2.2.
 // Thread t serves class cls(t) only (class-major allocation thr_start[]); accumulators persist over all
 // units of a channel and are flushed to `part0` / `partl` when the channel changes.
-template <typename T, int MAXT, int MINB, int TH>
+template <typename T, int MAXT, int MINB, int TH, int KT>
 __global__ void __launch_bounds__(MAXT, MINB)
 plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                    float *__restrict__ part0, float *__restrict__ partl /* level l at l*C*np*100 */,
@@ -1046,22 +1078,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) gsum += d[rr][cc];
                 }
-#pragma unroll
-                for (int rr = 0; rr < TH + 4; ++rr) {
-                    const float4 q0 = *reinterpret_cast<const float4 *>(ysrc + rr * pl);
-                    const float4 q1 = *reinterpret_cast<const float4 *>(ysrc + rr * pl + 4);
-                    const float in[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-#pragma unroll
-                    for (int uu = 0; uu < 5; ++uu) {
-                        const int dr = rr - uu;
-                        if (dr >= 0 && dr < TH) {
-#pragma unroll
-                            for (int v = 0; v < 5; ++v)
-#pragma unroll
-                                for (int cc = 0; cc < 4; ++cc) acc[uu * 5 + v] = fmaf(d[dr][cc], in[cc + v], acc[uu * 5 + v]);
-                        }
-                    }
-                }
+                wgrad_taps<TH, KT>(ysrc, pl, d, acc);
             }
         }
         __syncthreads();
@@ -1107,7 +1124,7 @@ plane_wgrad_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, cons
 //                    closed-form synthesis of Proposition 2 and the store of grad_x.
 // Used when a unit's item list fits one round of the block (<= 256 tiles); otherwise the separate weight-
 // gradient and input-gradient kernels run.
-template <typename T, int TH, int BULK>  // BULK: tensors prefetched by bulk copy (0 none, 2 x and grad_out)
+template <typename T, int TH, int BULK, int KT>  // BULK: tensors prefetched by bulk copy (0 none, 2 x and grad_out)
 __global__ void __launch_bounds__(256, 2)
 plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const T *__restrict__ go,
                  const float *__restrict__ w0, const float *__restrict__ s0, const float *__restrict__ wl,
@@ -1225,7 +1242,7 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
             if (TH == 4) {
                 float w[KK];
                 load_weights(sm + item.wt, w);
-                conv_tile<TH, true>(gsrc, pitch, w, acc, d);
+                conv_tile<TH, true, KT>(gsrc, pitch, w, acc, d);
             } else {
 #pragma unroll
                 for (int rr = 0; rr < TH; ++rr) {
@@ -1242,32 +1259,12 @@ plane_bwd_kernel(const __grid_constant__ Geom g, const T *__restrict__ x, const 
 #pragma unroll
                         for (int cc = 0; cc < 4; ++cc) gsum += d[rr][cc];
                 }
-                // the next window row is fetched while the current one is used
-                float4 n0 = *reinterpret_cast<const float4 *>(ysrc);
-                float4 n1 = *reinterpret_cast<const float4 *>(ysrc + 4);
-#pragma unroll
-                for (int rr = 0; rr < TH + 4; ++rr) {
-                    const float in[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
-                    if (rr + 1 < TH + 4) {
-                        n0 = *reinterpret_cast<const float4 *>(ysrc + (rr + 1) * pitch);
-                        n1 = *reinterpret_cast<const float4 *>(ysrc + (rr + 1) * pitch + 4);
-                    }
-#pragma unroll
-                    for (int uu = 0; uu < 5; ++uu) {
-                        const int dr = rr - uu;
-                        if (dr >= 0 && dr < TH) {
-#pragma unroll
-                            for (int v = 0; v < 5; ++v)
-#pragma unroll
-                                for (int cc = 0; cc < 4; ++cc) accw[uu * 5 + v] = fmaf(d[dr][cc], in[cc + v], accw[uu * 5 + v]);
-                        }
-                    }
-                }
+                wgrad_taps<TH, KT>(ysrc, pitch, d, accw);
             }
             if (TH != 4) {  // input gradient: rotated-kernel conv of the D window
                 float w[KK];
                 load_weights(sm + item.wt, w);
-                conv_tile<TH>(gsrc, pitch, w, acc);
+                conv_tile<TH, false, KT>(gsrc, pitch, w, acc);
             }
             if (item.z >= 0) {
                 const int zp = (item.meta >> 10) & 0x3ff, zleft = (item.meta >> 20) & 0xf;
@@ -1785,14 +1782,15 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
                        const float *sl, T *out, int *status, cudaStream_t st) {
     cudaError_t e;
     const size_t smem = (size_t)g.smem_floats * 4;
-#define WT_LAUNCH_FWD_TH(MAXT_, MINB_, TH_)                                                         \
+#define WT_LAUNCH_FWD_KT(MAXT_, MINB_, TH_, KT_)                                                    \
     {                                                                                               \
-        constexpr auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_, TH_>;                         \
+        constexpr auto kern = plane_fwd_kernel<T, FLIP, MAXT_, MINB_, TH_, KT_>;                    \
         if ((e = opt_in_smem<kern>()) != cudaSuccess) return e;                                     \
         if ((e = launch_overlapped(kern, (unsigned)g.nblocks, (unsigned)g.nthreads, smem, st, g, x, w0, s0, b0, wl, sl, \
                                    out, status)) != cudaSuccess)                                    \
             return e;                                                                               \
     }
+#define WT_LAUNCH_FWD_TH(MAXT_, MINB_, TH_) { if (g.taps == 3) WT_LAUNCH_FWD_KT(MAXT_, MINB_, TH_, 3) else WT_LAUNCH_FWD_KT(MAXT_, MINB_, TH_, 5) }
 #define WT_LAUNCH_FWD(MAXT_, MINB_) { if (g.th == 8) WT_LAUNCH_FWD_TH(MAXT_, MINB_, 8) else WT_LAUNCH_FWD_TH(MAXT_, MINB_, 4) }
     if (g.nthreads <= 128 && g.blocks_per_sm <= 3) {
         WT_LAUNCH_FWD(128, 3)
@@ -1803,6 +1801,7 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
     }
 #undef WT_LAUNCH_FWD
 #undef WT_LAUNCH_FWD_TH
+#undef WT_LAUNCH_FWD_KT
     return cudaGetLastError();
 }
 
@@ -1811,11 +1810,12 @@ cudaError_t launch_fwd(const Geom &g, const T *x, const float *w0, const float *
 template <typename T>
 cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *w0, const float *s0, const float *b0,
                     const float *wl, const float *sl, T *out, char *ws, cudaStream_t st, unsigned tag, unsigned tune = 0,
-                    bool no_copy = false) {
+                    bool no_copy = false, int taps = 5) {
     Geom g;
     if (!plan_forward(B, C, H, W, L, (int)sizeof(T), g, tune)) return cudaErrorInvalidValue;
     g.no_copy = no_copy;
     g.tag = tag;
+    g.taps = taps;
     return launch_fwd<T, false>(g, x, w0, s0, b0, wl, sl, out, reinterpret_cast<int *>(ws), st);
 }
 
@@ -1824,29 +1824,32 @@ cudaError_t forward(int B, int C, int H, int W, int L, const T *x, const float *
 template <typename T>
 cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go, const float *w0, const float *s0,
                      const float *wl, const float *sl, T *gx, char *ws, EpiloguePtrs *ep, cudaStream_t st, unsigned tag,
-                     unsigned tune = 0, bool no_copy = false) {
+                     unsigned tune = 0, bool no_copy = false, int taps = 5) {
     Geom gw, gf;
     cudaError_t e;
     if (plan_bwd_fused(B, C, H, W, L, (int)sizeof(T), gw, tune)) {
         gw.no_copy = no_copy;
         gw.tag = tag;
+        gw.taps = taps;
         float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
         float *partl = part0 + (size_t)C * gw.np * (KK + 1);
-#define WT_LAUNCH_BWD(TH_, BULK_)                                                                          \
+#define WT_LAUNCH_BWD_KT(TH_, BULK_, KT_)                                                                  \
     {                                                                                                      \
-        constexpr auto kb = plane_bwd_kernel<T, TH_, BULK_>;                                               \
+        constexpr auto kb = plane_bwd_kernel<T, TH_, BULK_, KT_>;                                          \
         if ((e = opt_in_smem<kb>()) != cudaSuccess) return e;                                              \
         if ((e = launch_overlapped(kb, (unsigned)gw.nblocks, (unsigned)gw.nthreads, (size_t)gw.smem_floats * 4, st, gw, \
                                    x, go, w0, s0, wl, sl, gx, part0, partl, reinterpret_cast<int *>(ws))) !=  \
             cudaSuccess)                                                                                   \
             return e;                                                                                      \
     }
+#define WT_LAUNCH_BWD(TH_, BULK_) { if (taps == 3) WT_LAUNCH_BWD_KT(TH_, BULK_, 3) else WT_LAUNCH_BWD_KT(TH_, BULK_, 5) }
         if (gw.th == 8) {
             if (gw.bulk == 2) WT_LAUNCH_BWD(8, 2) else WT_LAUNCH_BWD(8, 0)
         } else {
             if (gw.bulk == 2) WT_LAUNCH_BWD(4, 2) else WT_LAUNCH_BWD(4, 0)
         }
 #undef WT_LAUNCH_BWD
+#undef WT_LAUNCH_BWD_KT
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         ep->part0 = part0;
         ep->np0 = gw.np;
@@ -1861,24 +1864,27 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
         return cudaErrorInvalidValue;
     gw.no_copy = gf.no_copy = no_copy;
     gw.tag = gf.tag = tag;
+    gw.taps = gf.taps = taps;
     int *status = reinterpret_cast<int *>(ws);
     float *part0 = reinterpret_cast<float *>(ws + STATUS_BYTES);
     float *partl = part0 + (size_t)C * gw.np * (KK + 1);
     const size_t smem = (size_t)gw.smem_floats * 4;
-#define WT_LAUNCH_WG(MAXT_, MINB_, TH_)                                                            \
+#define WT_LAUNCH_WG_KT(MAXT_, MINB_, TH_, KT_)                                                    \
     {                                                                                              \
-        constexpr auto kw = plane_wgrad_kernel<T, MAXT_, MINB_, TH_>;                              \
+        constexpr auto kw = plane_wgrad_kernel<T, MAXT_, MINB_, TH_, KT_>;                         \
         if ((e = opt_in_smem<kw>()) != cudaSuccess) return e;                                      \
         if ((e = launch_overlapped(kw, (unsigned)gw.nblocks, (unsigned)gw.nthreads, smem, st, gw, x, go, part0, partl, \
                                    status)) != cudaSuccess)                                        \
             return e;                                                                              \
     }
+#define WT_LAUNCH_WG(MAXT_, MINB_, TH_) { if (taps == 3) WT_LAUNCH_WG_KT(MAXT_, MINB_, TH_, 3) else WT_LAUNCH_WG_KT(MAXT_, MINB_, TH_, 5) }
     if (gw.nthreads <= 128) {
         if (gw.th == 8) WT_LAUNCH_WG(128, 4, 8) else WT_LAUNCH_WG(128, 4, 4)
     } else {
         if (gw.th == 8) WT_LAUNCH_WG(256, 2, 8) else WT_LAUNCH_WG(256, 2, 4)
     }
 #undef WT_LAUNCH_WG
+#undef WT_LAUNCH_WG_KT
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = launch_fwd<T, true>(gf, go, w0, s0, nullptr, wl, sl, gx, status, st)) != cudaSuccess) return e;
     ep->part0 = part0;
@@ -1896,10 +1902,10 @@ cudaError_t backward(int B, int C, int H, int W, int L, const T *x, const T *go,
 #define WT_PLANE_INSTANTIATE(T, EXTERN)                                                                                    \
     EXTERN template cudaError_t forward<T>(int, int, int, int, int, const T *, const float *, const float *, const float *, \
                                            const float *, const float *, T *, char *, cudaStream_t, unsigned, unsigned,    \
-                                           bool);                                                                          \
+                                           bool, int);                                                                     \
     EXTERN template cudaError_t backward<T>(int, int, int, int, int, const T *, const T *, const float *, const float *,    \
                                             const float *, const float *, T *, char *, EpiloguePtrs *, cudaStream_t,       \
-                                            unsigned, unsigned, bool);
+                                            unsigned, unsigned, bool, int);
 
 }  // namespace plane
 }  // namespace wt

@@ -179,9 +179,11 @@ __global__ void extract_k3_kernel(const float *__restrict__ ae, const float *__r
     else b[(f - nf0) * 9 + t] = be[(f - nf0) * 25 + u * 5 + v];
 }
 
+// `taps` (k = 5 only): 3 when the tables hold 3 x 3 kernels with a zero border; the block-per-plane kernels then
+// leave the border out of their loops, the other kernel families multiply through it.
 template <typename T, int K>
 wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, const float *s0, const float *b0,
-                         const float *wl, const float *sl, void *out, char *ws, cudaStream_t st) {
+                         const float *wl, const float *sl, void *out, char *ws, cudaStream_t st, int taps = 5) {
     if (use_ref_chain(d)) return wt::refchain::forward<T, K>(d, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws, st);
     if constexpr (K == 3) {
         if (use_k3_embedding(d)) {
@@ -191,7 +193,7 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
             const size_t n = (e.nf0 + e.nfl) * 25;
             embed_k3_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w0, wl, w0e, wle, e.nf0, e.nfl);
             if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
-            return forward_tk<T, 5>(&d5, x, w0e, s0, b0, wle, sl, out, ws + e.inner, st);
+            return forward_tk<T, 5>(&d5, x, w0e, s0, b0, wle, sl, out, ws + e.inner, st, 3);
         }
     }
     if constexpr (K == 5) {
@@ -213,7 +215,7 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
         if constexpr (K == 5)
             return wt::plane::forward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, w0, s0, b0, wl, sl, (T *)out, ws,
                                          st, next_status_tag(), d->flags >> 8,
-                                         (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) == cudaSuccess
+                                         (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, taps) == cudaSuccess
                        ? WTCONV_OK
                        : WTCONV_ERR_CUDA;
     }
@@ -223,7 +225,7 @@ wtconv_status forward_tk(const wtconv_desc *d, const void *x, const float *w0, c
 template <typename T, int K>
 wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, const float *w0, const float *s0,
                           const float *b0, const float *wl, const float *sl, void *gx, float *gw0, float *gs0,
-                          float *gb0, float *gwl, float *gsl, char *ws, cudaStream_t st) {
+                          float *gb0, float *gwl, float *gsl, char *ws, cudaStream_t st, int taps = 5) {
     if (use_ref_chain(d))
         return wt::refchain::backward<T, K>(d, (const T *)x, (const T *)g, w0, s0, b0, wl, sl, (T *)gx, gw0, gs0, gb0, gwl, gsl,
                                             ws, st);
@@ -235,7 +237,7 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
             const size_t n = (e.nf0 + e.nfl) * 25, n3 = (e.nf0 + e.nfl) * 9;
             embed_k3_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(w0, wl, w0e, wle, e.nf0, e.nfl);
             if (launch_status() != WTCONV_OK) return WTCONV_ERR_CUDA;
-            const wtconv_status st5 = backward_tk<T, 5>(&d5, x, g, w0e, s0, b0, wle, sl, gx, gw0e, gs0, gb0, gwle, gsl, ws + e.inner, st);
+            const wtconv_status st5 = backward_tk<T, 5>(&d5, x, g, w0e, s0, b0, wle, sl, gx, gw0e, gs0, gb0, gwle, gsl, ws + e.inner, st, 3);
             if (st5 != WTCONV_OK) return st5;
             extract_k3_kernel<<<(unsigned)((n3 + 255) / 256), 256, 0, st>>>(gw0e, gwle, gw0, gwl, e.nf0, e.nfl);
             return launch_status();
@@ -265,7 +267,7 @@ wtconv_status backward_tk(const wtconv_desc *d, const void *x, const void *g, co
             wt::EpiloguePtrs ep = {};
             if (wt::plane::backward<T>(d->B, d->C, d->H, d->W, d->L, (const T *)x, (const T *)g, w0, s0, wl, sl,
                                        (T *)gx, ws, &ep, st, next_status_tag(), d->flags >> 8,
-                                       (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0) != cudaSuccess)
+                                       (d->flags & WTCONV_FLAG_TEST_NO_COPY) != 0, taps) != cudaSuccess)
                 return WTCONV_ERR_CUDA;
             return launch_epilogue(d, ep, w0, s0, b0, wl, sl, gw0, gs0, gb0, gwl, gsl, st);
         }
