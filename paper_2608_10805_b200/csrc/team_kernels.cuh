@@ -542,8 +542,6 @@ inline bool plan_th(int B, int C, int H, int W, int L, int eb, bool bwd, int TH,
         g.ty[l] = (g.Hl[l] + TH - 1) / TH;
         g.rows[l] = g.ty[l] * TH + 4;
         g.pitch[l] = g.tx[l] * 4 + 4;
-        g.sub[l] = g.rows[l] * g.pitch[l];
-        while ((g.sub[l] / 4) % 8 != 2) g.sub[l] += 4;  // subbands 2 chunks (mod 8) apart: neighbouring subband tiles hit different banks
         if (l) useful += 4.0 * g.Hl[l] * g.Wl[l];
     }
     g.nbase = g.tx[0] * g.ty[0];
@@ -551,10 +549,19 @@ inline bool plan_th(int B, int C, int H, int W, int L, int eb, bool bwd, int TH,
     for (int l = 1; l <= L; ++l) g.lvl_start[l + 1] = g.lvl_start[l] + 4 * g.tx[l] * g.ty[l];
     g.ntiles = g.nbase + g.lvl_start[L + 1];
     if (g.ntiles > 64) return false;
-    int off = 0;
-    for (int l = 0; l <= L; ++l) { g.offA[l] = off; off += (l ? 4 : 1) * g.sub[l]; }
-    for (int l = 0; l <= L; ++l) { g.offG[l] = off; if (bwd) off += (l ? 4 : 1) * g.sub[l]; }
-    const int slot_min = pad4(off);
+    // Array layout of one plane slot.  With fewer than 8 planes per unit a quarter-warp holds several tiles of one
+    // plane, and the subbands are put 2 chunks (mod 8) apart so that neighbouring subband tiles hit different banks;
+    // with 8 or more it holds the same tile of 8 planes and only the slot stride matters (no padding: more teams fit).
+    auto layout = [&](TGeom &t, bool pad_subbands) {
+        for (int l = 0; l <= L; ++l) {
+            t.sub[l] = t.rows[l] * t.pitch[l];
+            while (pad_subbands && (t.sub[l] / 4) % 8 != 2) t.sub[l] += 4;
+        }
+        int off = 0;
+        for (int l = 0; l <= L; ++l) { t.offA[l] = off; off += (l ? 4 : 1) * t.sub[l]; }
+        for (int l = 0; l <= L; ++l) { t.offG[l] = off; if (bwd) off += (l ? 4 : 1) * t.sub[l]; }
+        return pad4(off);
+    };
     g.HW = H * W;
     g.plane_bytes = H * W * eb;
     g.vec2 = (W % 2 == 0) ? 1 : 0;
@@ -579,7 +586,7 @@ inline bool plan_th(int B, int C, int H, int W, int L, int eb, bool bwd, int TH,
         TGeom c = g;
         c.G = G; c.T = T; c.team = team; c.d_G = make_fastdiv(G);
         // plane slots 8 / min(G, 8) chunks (mod 8) apart: a quarter-warp = the same tiles of min(G, 8) planes, bank-conflict free
-        c.slot_floats = slot_min;
+        c.slot_floats = layout(c, G < 8);
         const int want = G >= 8 ? 1 : 8 / G;
         while (G > 1 && (c.slot_floats / 4) % 8 != want % 8) c.slot_floats += 4;
         c.unit_bytes = G * g.plane_bytes;
